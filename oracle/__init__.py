@@ -1,0 +1,209 @@
+"""ctypes front end of the double-precision CPU oracle (``bns_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the benchmark's CPU-baseline
+leg.  It has no dependency on the CUDA library and the CUDA library has none on it.
+
+All tensors are numpy arrays in NCHW.  Activations and gradients are passed as float32 (bf16 data
+is widened exactly before the call); every result is float64.
+"""
+from __future__ import annotations
+
+import ctypes
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import numpy as np
+
+from .build import build as _build
+
+RULE_FULL, RULE_BATCH, RULE_FEATURE, RULE_VIRTUAL = 0, 1, 2, 3
+OFFSETS_SHARED, OFFSETS_PER_SAMPLE, OFFSETS_PER_MAP = 0, 1, 2
+
+
+class _CSampling(ctypes.Structure):
+    _fields_ = [
+        ("rule", ctypes.c_int),
+        ("k", ctypes.c_int),
+        ("sample_idx", ctypes.c_void_p),
+        ("ph", ctypes.c_int),
+        ("pw", ctypes.c_int),
+        ("offset_mode", ctypes.c_int),
+        ("offsets", ctypes.c_void_p),
+        ("nv", ctypes.c_int),
+    ]
+
+
+@dataclass
+class Sampling:
+    """Which elements enter the statistics (Eq. 3): the paper's S."""
+    rule: int = RULE_FULL
+    sample_idx: Optional[np.ndarray] = None   # BATCH: int32 [k]
+    ph: int = 0                               # FEATURE
+    pw: int = 0
+    offset_mode: int = OFFSETS_SHARED
+    offsets: Optional[np.ndarray] = None      # FEATURE: int32 [1|N|N*C, 2]
+    nv: int = 0                               # VIRTUAL
+
+    @staticmethod
+    def full():
+        return Sampling(RULE_FULL)
+
+    @staticmethod
+    def batch(sample_idx):
+        return Sampling(RULE_BATCH, sample_idx=np.ascontiguousarray(sample_idx, dtype=np.int32))
+
+    @staticmethod
+    def feature(ph, pw, offsets, offset_mode=OFFSETS_SHARED):
+        off = np.ascontiguousarray(offsets, dtype=np.int32).reshape(-1, 2)
+        return Sampling(RULE_FEATURE, ph=int(ph), pw=int(pw), offset_mode=int(offset_mode), offsets=off)
+
+    @staticmethod
+    def virtual(nv):
+        return Sampling(RULE_VIRTUAL, nv=int(nv))
+
+    def _c(self):
+        keep = []
+        c = _CSampling()
+        c.rule = self.rule
+        if self.rule == RULE_BATCH:
+            idx = np.ascontiguousarray(self.sample_idx, dtype=np.int32)
+            keep.append(idx)
+            c.k = idx.size
+            c.sample_idx = idx.ctypes.data
+        if self.rule == RULE_FEATURE:
+            off = np.ascontiguousarray(self.offsets, dtype=np.int32)
+            keep.append(off)
+            c.ph, c.pw, c.offset_mode = self.ph, self.pw, self.offset_mode
+            c.offsets = off.ctypes.data
+        c.nv = self.nv
+        return c, keep
+
+
+_lib = None
+
+
+def _library():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(_build())
+        lib.oracle_sample_count.restype = ctypes.c_longlong
+        lib.oracle_adder_tree_depth_ratio.restype = ctypes.c_double
+        lib.oracle_forward.restype = None
+        lib.oracle_backward.restype = None
+        lib.oracle_selection_mask.restype = None
+        _lib = lib
+    return _lib
+
+
+def _f32(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _ptr(a):
+    return ctypes.c_void_p(None if a is None else a.ctypes.data)
+
+
+def _channels(channels, C):
+    if channels is None:
+        return None, C
+    ch = np.ascontiguousarray(channels, dtype=np.int32)
+    assert ch.ndim == 1 and ch.size > 0 and ch.min() >= 0 and ch.max() < C
+    return ch, int(ch.size)
+
+
+def _check_offsets(sp: Sampling, N, C, H, W):
+    if sp.rule == RULE_BATCH:
+        idx = sp.sample_idx
+        assert idx.size >= 1 and idx.min() >= 0 and idx.max() < N and np.unique(idx).size == idx.size
+    if sp.rule == RULE_FEATURE:
+        count = {OFFSETS_SHARED: 1, OFFSETS_PER_SAMPLE: N, OFFSETS_PER_MAP: N * C}[sp.offset_mode]
+        off = sp.offsets
+        assert off.shape == (count, 2)
+        assert 1 <= sp.ph <= H and 1 <= sp.pw <= W
+        assert off[:, 0].min() >= 0 and off[:, 0].max() <= H - sp.ph
+        assert off[:, 1].min() >= 0 and off[:, 1].max() <= W - sp.pw
+    if sp.rule == RULE_VIRTUAL:
+        assert sp.nv >= 1
+
+
+def sample_count(N, H, W, sp: Sampling) -> int:
+    c, _keep = sp._c()
+    return int(_library().oracle_sample_count(N, H, W, ctypes.byref(c)))
+
+
+def adder_tree_depth_ratio(N, H, W, sp: Sampling) -> float:
+    c, _keep = sp._c()
+    return float(_library().oracle_adder_tree_depth_ratio(N, H, W, ctypes.byref(c)))
+
+
+def selection_mask(N, C, H, W, sp: Sampling) -> np.ndarray:
+    _check_offsets(sp, N, C, H, W)
+    c, _keep = sp._c()
+    mask = np.zeros((N, C, H, W), dtype=np.uint8)
+    _library().oracle_selection_mask(N, C, H, W, ctypes.byref(c), _ptr(mask))
+    return mask
+
+
+@dataclass
+class Forward:
+    y: Optional[np.ndarray]
+    yv: Optional[np.ndarray]
+    mean: np.ndarray
+    var: np.ndarray
+    invstd: np.ndarray
+
+
+@dataclass
+class Backward:
+    dx: Optional[np.ndarray]
+    dxv: Optional[np.ndarray]
+    dgamma: np.ndarray
+    dbeta: np.ndarray
+
+
+def forward(x, gamma, beta, eps, sp: Sampling, xv=None, channels: Optional[Sequence[int]] = None,
+            want_y=True, want_yv=True) -> Forward:
+    """Eq. 1 with the statistics of Eq. 3 (Eq. 2 for the FULL rule), for the listed channels."""
+    x = _f32(x)
+    N, C, H, W = x.shape
+    _check_offsets(sp, N, C, H, W)
+    xv = _f32(xv)
+    if sp.rule == RULE_VIRTUAL:
+        assert xv is not None and xv.shape == (sp.nv, C, H, W)
+    gamma, beta = _f32(gamma), _f32(beta)
+    assert gamma.shape == (C,) and beta.shape == (C,) and eps > 0
+    ch, nch = _channels(channels, C)
+    y = np.empty((N, nch, H, W), dtype=np.float64) if want_y else None
+    yv = np.empty((sp.nv, nch, H, W), dtype=np.float64) if (sp.rule == RULE_VIRTUAL and want_yv) else None
+    mean, var, invstd = (np.empty(nch, dtype=np.float64) for _ in range(3))
+    c, _keep = sp._c()
+    _library().oracle_forward(N, C, H, W, _ptr(x), _ptr(xv), _ptr(gamma), _ptr(beta), ctypes.c_double(eps),
+                              ctypes.byref(c), _ptr(ch), nch, _ptr(y), _ptr(yv), _ptr(mean), _ptr(var),
+                              _ptr(invstd))
+    return Forward(y, yv, mean, var, invstd)
+
+
+def backward(x, dy, gamma, mean, var, eps, sp: Sampling, xv=None, dyv=None,
+             channels: Optional[Sequence[int]] = None, want_dx=True, want_dxv=True) -> Backward:
+    """Eq. 5 / Eq. 6 for the listed channels; ``mean`` and ``var`` are ``forward``'s for those channels."""
+    x, dy = _f32(x), _f32(dy)
+    N, C, H, W = x.shape
+    assert dy.shape == x.shape
+    _check_offsets(sp, N, C, H, W)
+    xv, dyv = _f32(xv), _f32(dyv)
+    if sp.rule == RULE_VIRTUAL:
+        assert xv is not None and xv.shape == (sp.nv, C, H, W)
+        assert dyv is None or dyv.shape == xv.shape
+    gamma = _f32(gamma)
+    ch, nch = _channels(channels, C)
+    mean = np.ascontiguousarray(mean, dtype=np.float64)
+    var = np.ascontiguousarray(var, dtype=np.float64)
+    assert mean.shape == (nch,) and var.shape == (nch,)
+    dx = np.empty((N, nch, H, W), dtype=np.float64) if want_dx else None
+    dxv = np.empty((sp.nv, nch, H, W), dtype=np.float64) if (sp.rule == RULE_VIRTUAL and want_dxv) else None
+    dgamma, dbeta = (np.empty(nch, dtype=np.float64) for _ in range(2))
+    c, _keep = sp._c()
+    _library().oracle_backward(N, C, H, W, _ptr(x), _ptr(xv), _ptr(dy), _ptr(dyv), _ptr(gamma), _ptr(mean),
+                               _ptr(var), ctypes.c_double(eps), ctypes.byref(c), _ptr(ch), nch, _ptr(dx),
+                               _ptr(dxv), _ptr(dgamma), _ptr(dbeta))
+    return Backward(dx, dxv, dgamma, dbeta)
