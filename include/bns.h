@@ -1,0 +1,187 @@
+/*
+ * bns.h - C ABI of the Batch Normalization Sampling library for NVIDIA B200 (sm_100a).
+ *
+ * One BN layer over a dense NCHW activation tensor whose per-channel mean and variance are
+ * estimated from a sampled subset S of the activations (arXiv 1810.10962, "Batch Normalization
+ * Sampling"), while normalise+affine and its gradient still cover the whole tensor.
+ *
+ * Conventions that hold for every entry point
+ *  - DEVICE pointers unless a comment says HOST.  The caller owns every buffer; the library
+ *    allocates no memory, keeps no state between calls (except the optional profiling hooks at
+ *    the end of this file) and never synchronises the host: all work is enqueued on `cuda_stream`
+ *    (a cudaStream_t passed as void*; NULL is the default stream).
+ *  - x, y, dy, dx share one shape and element type (`bns_shape`), are dense NCHW and 16-byte
+ *    aligned.  gamma, beta, mean, invstd, dgamma, dbeta are float[C].  Statistics and parameter
+ *    gradients are always fp32; bf16 tensors are rounded to nearest-even on store.
+ *  - Outputs must not alias inputs.
+ *  - Arguments are validated on the host before anything is launched; a negative status means
+ *    that nothing was enqueued.  No exception crosses this boundary.
+ *  - Results are a deterministic function of the inputs: no floating-point atomics are used and
+ *    every cross-block combine runs in a fixed order, so two runs give identical bits.
+ *  - `workspace` is scratch of at least bns_workspace_bytes() bytes, 256-byte aligned.  Calls that
+ *    overlap in time on the GPU need distinct workspaces.
+ */
+#ifndef BNS_H
+#define BNS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BNS_OK = 0,
+    BNS_ERR_NULL = -1,       /* a required pointer is NULL                                   */
+    BNS_ERR_SHAPE = -2,      /* non-positive or overflowing dimension, eps <= 0              */
+    BNS_ERR_RULE = -3,       /* unknown rule / offset mode, or a rule field out of range     */
+    BNS_ERR_INDEX = -4,      /* sample index or patch offset outside the tensor, or repeated */
+    BNS_ERR_DTYPE = -5,      /* unknown element type                                         */
+    BNS_ERR_ALIGN = -6,      /* a tensor pointer is not 16-byte aligned                      */
+    BNS_ERR_WORKSPACE = -7,  /* workspace NULL, misaligned or too small                      */
+    BNS_ERR_CUDA = -8        /* a CUDA runtime call failed (launch, copy)                    */
+} bns_status;
+
+typedef enum { BNS_F32 = 0, BNS_BF16 = 1 } bns_dtype;
+
+/* How the sampled set S is chosen (Sec. 4.1, Sec. 4.2 and Algorithms 1-3 of the paper). */
+typedef enum {
+    BNS_RULE_FULL = 0,     /* S = every element: ordinary BN (Eq. 2)                            */
+    BNS_RULE_BATCH = 1,    /* Batch Sampling: all elements of k chosen samples (Algorithm 1);   */
+                           /* Naive Sampling is the same rule with indices 0..k-1               */
+    BNS_RULE_FEATURE = 2,  /* Feature Sampling: one ph x pw patch of every feature map (Alg. 2) */
+    BNS_RULE_VIRTUAL = 3   /* Virtual Dataset Normalization: statistics from nv virtual samples */
+                           /* only (Algorithm 3); they are passed as a separate tensor xv       */
+} bns_rule;
+
+typedef enum {
+    BNS_OFF_SHARED = 0,      /* one (oh,ow) for the whole layer: the paper's rule (Sec. 4.1)  */
+    BNS_OFF_PER_SAMPLE = 1,  /* one (oh,ow) per sample n                                      */
+    BNS_OFF_PER_MAP = 2      /* one (oh,ow) per feature map (n,c), index n*C + c              */
+} bns_offset_mode;
+
+typedef struct {
+    int rule;                   /* bns_rule                                                       */
+    /* BATCH */
+    int k;                      /* number of sampled samples, 1..N                                */
+    const int32_t* sample_idx;  /* HOST, k distinct values in [0,N), any order; copied during the */
+                                /* call, so it may be reused as soon as the call returns          */
+    /* FEATURE */
+    int ph, pw;                 /* patch size, 1..H and 1..W                                      */
+    int offset_mode;            /* bns_offset_mode                                                */
+    const int32_t* offsets;     /* (oh,ow) int32 pairs, oh in [0,H-ph], ow in [0,W-pw]:           */
+                                /* SHARED: HOST, 1 pair (validated on the host);                  */
+                                /* PER_SAMPLE: DEVICE, N pairs; PER_MAP: DEVICE, N*C pairs.       */
+                                /* Device-resident pairs are checked by the kernels: a pair out   */
+                                /* of range is clamped into range and BNS_FLAG_BAD_OFFSET is set  */
+                                /* in the workspace status word (see bns_workspace_status)        */
+    /* VIRTUAL */
+    int nv;                     /* number of virtual samples, >= 1                                */
+    int xv_dtype;               /* bns_dtype of xv, yv, dyv, dxv                                  */
+    const void* xv;             /* [nv,C,H,W], 16-byte aligned                                    */
+    void* yv;                   /* forward: normalised virtual samples, may be NULL               */
+    const void* dyv;            /* backward: gradient reaching yv, may be NULL (treated as zeros) */
+    void* dxv;                  /* backward: gradient of xv, may be NULL                          */
+} bns_sampling;
+
+typedef struct {
+    int N, C, H, W;
+    int dtype;                  /* bns_dtype of x, y, dy, dx */
+} bns_shape;
+
+/* Scratch size that serves bns_forward, bns_backward and bns_full_bn for this shape and rule.
+ * Returns 0 if the arguments are invalid. */
+size_t bns_workspace_bytes(const bns_shape* shape, const bns_sampling* sampling);
+
+/*
+ * Forward (Eq. 1 with the sampled statistics of Eq. 3).
+ *   mean_c   = (1/s) sum_{i in S_c} x_i
+ *   var_c    = (1/s) sum_{i in S_c} (x_i - mean_c)^2            (biased)
+ *   invstd_c = 1 / sqrt(var_c + eps)
+ *   y_i      = gamma_c (x_i - mean_c) invstd_c + beta_c          for EVERY element of x
+ * VIRTUAL: S_c is all of xv[:,c,:,:]; yv (if not NULL) receives the same map applied to xv.
+ * Writes y, mean[C], invstd[C] (the statistics that the backward call needs).
+ */
+bns_status bns_forward(const bns_shape* shape, const void* x, const float* gamma, const float* beta,
+                       float eps, const bns_sampling* sampling, void* y, float* mean, float* invstd,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward (Eq. 5 with the modification of Eq. 6).  mean and invstd are the forward's outputs.
+ *   dbeta_c  = sum_i dy_i                      dgamma_c = sum_i dy_i xhat_i
+ * where both sums run over every element that was normalised with these statistics (all
+ * N*H*W real points, plus the virtual rows when dyv is given) - they keep their full length
+ * (Appendix C.1, "Speedup in the Backward Pass"), and
+ *   dx_i = gamma_c invstd_c ( dy_i - [i in S_c] (dbeta_c + xhat_i dgamma_c) / s )
+ * which is Eq. 6 with dl/dE and dl/dVar of Eq. 5 substituted.  VIRTUAL: no real element is in S;
+ * dxv (if not NULL) gets the upper branch for every virtual element.  rule FULL gives the
+ * ordinary BN backward.
+ */
+bns_status bns_backward(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
+                        const float* mean, const float* invstd, const bns_sampling* sampling,
+                        void* dx, float* dgamma, float* dbeta,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Ordinary BN forward (Eq. 1 with Eq. 2): the in-library comparison.  Same as bns_forward with
+ * rule FULL; its backward is bns_backward with rule FULL. */
+bns_status bns_full_bn(const bns_shape* shape, const void* x, const float* gamma, const float* beta,
+                       float eps, void* y, float* mean, float* invstd,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Forward and backward of one layer with HOST buffers for the large tensors: copies x and dy to
+ * the device, runs bns_forward and bns_backward, copies y, dx, mean, invstd, dgamma, dbeta back.
+ * x, dy, y, dx, gamma, beta and the six outputs are HOST pointers (pinned memory lets the copies
+ * run asynchronously); pointers inside `sampling` keep the meaning documented above.
+ * `arena` is DEVICE scratch of at least bns_host_arena_bytes() bytes, 256-byte aligned.
+ * Everything is enqueued on `cuda_stream`; synchronise it before reading the outputs.
+ * The paper has no counterpart (its measurements include input pipelines only as a whole).
+ */
+size_t bns_host_arena_bytes(const bns_shape* shape, const bns_sampling* sampling);
+bns_status bns_forward_backward_host(const bns_shape* shape, const void* x, const void* dy,
+                                     const float* gamma, const float* beta, float eps,
+                                     const bns_sampling* sampling, void* y, void* dx, float* mean,
+                                     float* invstd, float* dgamma, float* dbeta,
+                                     void* arena, size_t arena_bytes, void* cuda_stream);
+
+/* Test aid for the selection rule (Algorithms 1-3): writes 1 where the real element is in S and 0
+ * elsewhere; mask is uint8 [N,C,H,W] (all zeros for VIRTUAL).  Needs the same workspace. */
+bns_status bns_debug_selection_mask(const bns_shape* shape, const bns_sampling* sampling, uint8_t* mask,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Status word that kernels set in a workspace: synchronises the stream and copies it to *flags
+ * (HOST).  Every forward/backward/mask call clears the word first. */
+#define BNS_FLAG_BAD_OFFSET 1u /* a device-resident patch offset was outside [0,H-ph] x [0,W-pw] */
+bns_status bns_workspace_status(const void* workspace, uint32_t* flags, void* cuda_stream);
+
+const char* bns_status_string(bns_status status);
+
+/* ---- measurement hooks (process-wide, not thread-safe; off by default) ---------------------- */
+typedef enum {
+    BNS_KERNEL_COL_MOMENTS = 0,   /* statistics over whole samples (FULL, BATCH, VIRTUAL)       */
+    BNS_KERNEL_PATCH_MOMENTS = 1, /* statistics over patches (FEATURE)                          */
+    BNS_KERNEL_FINALIZE_STATS = 2,
+    BNS_KERNEL_NORMALIZE = 3,     /* y = a x + b over the whole tensor                          */
+    BNS_KERNEL_BWD_REDUCE = 4,    /* reads dy, x; writes dx = gamma invstd dy; partial sums     */
+    BNS_KERNEL_FINALIZE_BWD = 5,
+    BNS_KERNEL_COL_FIXUP = 6,     /* gradient with the statistics terms over whole samples      */
+    BNS_KERNEL_PATCH_FIXUP = 7,   /* the same over patches                                      */
+    BNS_KERNEL_MASK = 8,
+    BNS_KERNEL_KINDS = 9
+} bns_kernel_kind;
+
+/* Number of kernels this library has launched in this process since load (or since reset). */
+uint64_t bns_launch_count(void);
+void bns_launch_count_reset(void);
+/* With profiling on, every launch is bracketed by CUDA events on its own stream (up to a fixed
+ * pool; later launches go untimed).  bns_profile_read synchronises the recorded events and returns
+ * the launches and the summed device time of one kernel kind since the last bns_profile_enable. */
+void bns_profile_enable(int on);
+bns_status bns_profile_read(int kernel_kind, int* launches, float* total_ms);
+const char* bns_kernel_name(int kernel_kind);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BNS_H */

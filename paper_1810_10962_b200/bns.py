@@ -1,0 +1,339 @@
+"""Python binding of the C ABI in ``include/bns.h``.
+
+Argument marshalling only: every function hands raw device pointers, sizes and the current CUDA
+stream to ``libbns.so``; all arithmetic runs in that library's kernels.  PyTorch provides device
+memory and streams.  There is no fallback: if the library cannot be loaded, or a tensor is not a
+CUDA tensor, the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+OK = 0
+F32, BF16 = 0, 1
+RULE_FULL, RULE_BATCH, RULE_FEATURE, RULE_VIRTUAL = 0, 1, 2, 3
+OFF_SHARED, OFF_PER_SAMPLE, OFF_PER_MAP = 0, 1, 2
+FLAG_BAD_OFFSET = 1
+
+KERNEL_KINDS = 9
+(KERNEL_COL_MOMENTS, KERNEL_PATCH_MOMENTS, KERNEL_FINALIZE_STATS, KERNEL_NORMALIZE, KERNEL_BWD_REDUCE,
+ KERNEL_FINALIZE_BWD, KERNEL_COL_FIXUP, KERNEL_PATCH_FIXUP, KERNEL_MASK) = range(KERNEL_KINDS)
+
+EXPORTS = [
+    "bns_workspace_bytes", "bns_forward", "bns_backward", "bns_full_bn", "bns_host_arena_bytes",
+    "bns_forward_backward_host", "bns_debug_selection_mask", "bns_workspace_status", "bns_status_string",
+    "bns_launch_count", "bns_launch_count_reset", "bns_profile_enable", "bns_profile_read", "bns_kernel_name",
+]
+
+
+class BnsError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+        self.status = status
+
+
+class _Shape(ctypes.Structure):
+    _fields_ = [("N", ctypes.c_int), ("C", ctypes.c_int), ("H", ctypes.c_int), ("W", ctypes.c_int),
+                ("dtype", ctypes.c_int)]
+
+
+class _Sampling(ctypes.Structure):
+    _fields_ = [
+        ("rule", ctypes.c_int), ("k", ctypes.c_int), ("sample_idx", ctypes.c_void_p),
+        ("ph", ctypes.c_int), ("pw", ctypes.c_int), ("offset_mode", ctypes.c_int), ("offsets", ctypes.c_void_p),
+        ("nv", ctypes.c_int), ("xv_dtype", ctypes.c_int), ("xv", ctypes.c_void_p), ("yv", ctypes.c_void_p),
+        ("dyv", ctypes.c_void_p), ("dxv", ctypes.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIBRARY
+
+
+def load():
+    """Load ``libbns.so`` (building it first if its sources are newer and nvcc is present)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if _build.is_stale():
+        try:
+            _build.build()
+        except Exception as exc:  # no compiler: only acceptable if a built library is already there
+            if not os.path.exists(_build.LIBRARY):
+                raise RuntimeError(f"libbns.so is missing and could not be built: {exc}") from exc
+    lib = ctypes.CDLL(_build.LIBRARY)
+    vp, sz, fl = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_float
+    shp, smp = ctypes.POINTER(_Shape), ctypes.POINTER(_Sampling)
+    lib.bns_workspace_bytes.restype = sz
+    lib.bns_workspace_bytes.argtypes = [shp, smp]
+    lib.bns_forward.restype = ctypes.c_int
+    lib.bns_forward.argtypes = [shp, vp, vp, vp, fl, smp, vp, vp, vp, vp, sz, vp]
+    lib.bns_backward.restype = ctypes.c_int
+    lib.bns_backward.argtypes = [shp, vp, vp, vp, vp, vp, smp, vp, vp, vp, vp, sz, vp]
+    lib.bns_full_bn.restype = ctypes.c_int
+    lib.bns_full_bn.argtypes = [shp, vp, vp, vp, fl, vp, vp, vp, vp, sz, vp]
+    lib.bns_host_arena_bytes.restype = sz
+    lib.bns_host_arena_bytes.argtypes = [shp, smp]
+    lib.bns_forward_backward_host.restype = ctypes.c_int
+    lib.bns_forward_backward_host.argtypes = [shp, vp, vp, vp, vp, fl, smp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.bns_debug_selection_mask.restype = ctypes.c_int
+    lib.bns_debug_selection_mask.argtypes = [shp, smp, vp, vp, sz, vp]
+    lib.bns_workspace_status.restype = ctypes.c_int
+    lib.bns_workspace_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+    lib.bns_status_string.restype = ctypes.c_char_p
+    lib.bns_status_string.argtypes = [ctypes.c_int]
+    lib.bns_launch_count.restype = ctypes.c_uint64
+    lib.bns_launch_count_reset.restype = None
+    lib.bns_profile_enable.restype = None
+    lib.bns_profile_enable.argtypes = [ctypes.c_int]
+    lib.bns_profile_read.restype = ctypes.c_int
+    lib.bns_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float)]
+    lib.bns_kernel_name.restype = ctypes.c_char_p
+    lib.bns_kernel_name.argtypes = [ctypes.c_int]
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().bns_status_string(int(status)).decode()
+
+
+# ----------------------------------------------------------------------------- sampling rule
+@dataclass
+class Sampling:
+    """The sampled set S.  ``sample_idx`` is a host int32 array; ``offsets`` is a host array for the
+    shared location and a CUDA int32 tensor [N,2] / [N*C,2] otherwise; xv, yv, dyv, dxv are CUDA
+    tensors [nv,C,H,W]."""
+    rule: int = RULE_FULL
+    sample_idx: Optional[np.ndarray] = None
+    ph: int = 0
+    pw: int = 0
+    offset_mode: int = OFF_SHARED
+    offsets: object = None
+    nv: int = 0
+    xv: Optional[torch.Tensor] = None
+    yv: Optional[torch.Tensor] = None
+    dyv: Optional[torch.Tensor] = None
+    dxv: Optional[torch.Tensor] = None
+
+    @staticmethod
+    def full():
+        return Sampling(RULE_FULL)
+
+    @staticmethod
+    def batch(sample_idx):
+        return Sampling(RULE_BATCH, sample_idx=np.ascontiguousarray(sample_idx, dtype=np.int32))
+
+    @staticmethod
+    def feature(ph, pw, offsets, offset_mode=OFF_SHARED):
+        if offset_mode == OFF_SHARED:
+            offsets = np.ascontiguousarray(np.asarray(offsets).reshape(-1), dtype=np.int32)
+        return Sampling(RULE_FEATURE, ph=int(ph), pw=int(pw), offset_mode=int(offset_mode), offsets=offsets)
+
+    @staticmethod
+    def virtual(xv, yv=None, dyv=None, dxv=None):
+        return Sampling(RULE_VIRTUAL, nv=int(xv.shape[0]), xv=xv, yv=yv, dyv=dyv, dxv=dxv)
+
+    def _c(self) -> _Sampling:
+        c = _Sampling()
+        c.rule = self.rule
+        if self.rule == RULE_BATCH:
+            c.k = int(self.sample_idx.size)
+            c.sample_idx = self.sample_idx.ctypes.data
+        elif self.rule == RULE_FEATURE:
+            c.ph, c.pw, c.offset_mode = self.ph, self.pw, self.offset_mode
+            if self.offset_mode == OFF_SHARED:
+                c.offsets = self.offsets.ctypes.data
+            else:
+                off = self.offsets
+                if not (isinstance(off, torch.Tensor) and off.is_cuda and off.dtype == torch.int32 and off.is_contiguous()):
+                    raise TypeError("per-sample / per-map offsets must be a contiguous CUDA int32 tensor")
+                c.offsets = off.data_ptr()
+        elif self.rule == RULE_VIRTUAL:
+            c.nv = self.nv
+            c.xv_dtype = _dtype_code(self.xv)
+            c.xv = _dev(self.xv)
+            for name in ("yv", "dyv", "dxv"):
+                t = getattr(self, name)
+                if t is not None:
+                    if t.dtype != self.xv.dtype or t.shape != self.xv.shape:
+                        raise TypeError(f"{name} must match xv in dtype and shape")
+                    setattr(c, name, _dev(t))
+        return c
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported element type {t.dtype}")
+
+
+def _dev(t: torch.Tensor) -> int:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("expected a CUDA tensor (this library has no CPU path)")
+    if not t.is_contiguous():
+        raise TypeError("expected a contiguous tensor")
+    return t.data_ptr()
+
+
+def _vec(t: torch.Tensor, C: int) -> int:
+    if t.dtype != torch.float32 or t.numel() != C:
+        raise TypeError("per-channel vectors must be float32 of length C")
+    return _dev(t)
+
+
+def _shape(x: torch.Tensor) -> _Shape:
+    if x.dim() != 4:
+        raise TypeError("expected an NCHW tensor")
+    N, C, H, W = x.shape
+    return _Shape(N, C, H, W, _dtype_code(x))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(status: int, what: str):
+    if status != OK:
+        raise BnsError(status, what)
+
+
+def workspace_bytes(x: torch.Tensor, sampling: Sampling) -> int:
+    sh, sp = _shape(x), sampling._c()
+    n = load().bns_workspace_bytes(ctypes.byref(sh), ctypes.byref(sp))
+    if n == 0:
+        raise BnsError(-3, "bns_workspace_bytes (invalid shape or sampling rule)")
+    return int(n)
+
+
+def new_workspace(x: torch.Tensor, sampling: Sampling) -> torch.Tensor:
+    return torch.empty(workspace_bytes(x, sampling), dtype=torch.uint8, device=x.device)
+
+
+def _workspace(x, sampling, workspace):
+    if workspace is None:
+        workspace = new_workspace(x, sampling)
+    return workspace, workspace.data_ptr(), workspace.numel()
+
+
+# ----------------------------------------------------------------------------- the three calls
+def forward(x, gamma, beta, eps, sampling: Sampling, y=None, mean=None, invstd=None, workspace=None):
+    """bns_forward: returns (y, mean, invstd)."""
+    sh, sp = _shape(x), sampling._c()
+    C = x.shape[1]
+    y = torch.empty_like(x) if y is None else y
+    mean = torch.empty(C, dtype=torch.float32, device=x.device) if mean is None else mean
+    invstd = torch.empty(C, dtype=torch.float32, device=x.device) if invstd is None else invstd
+    ws, wp, wn = _workspace(x, sampling, workspace)
+    st = load().bns_forward(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), ctypes.byref(sp),
+                            _dev(y), _vec(mean, C), _vec(invstd, C), wp, wn, _stream())
+    _check(st, "bns_forward")
+    return y, mean, invstd
+
+
+def backward(x, dy, gamma, mean, invstd, sampling: Sampling, dx=None, dgamma=None, dbeta=None, workspace=None):
+    """bns_backward: returns (dx, dgamma, dbeta)."""
+    sh, sp = _shape(x), sampling._c()
+    C = x.shape[1]
+    if dy.shape != x.shape or dy.dtype != x.dtype:
+        raise TypeError("dy must match x")
+    dx = torch.empty_like(x) if dx is None else dx
+    dgamma = torch.empty(C, dtype=torch.float32, device=x.device) if dgamma is None else dgamma
+    dbeta = torch.empty(C, dtype=torch.float32, device=x.device) if dbeta is None else dbeta
+    ws, wp, wn = _workspace(x, sampling, workspace)
+    st = load().bns_backward(ctypes.byref(sh), _dev(x), _dev(dy), _vec(gamma, C), _vec(mean, C), _vec(invstd, C),
+                             ctypes.byref(sp), _dev(dx), _vec(dgamma, C), _vec(dbeta, C), wp, wn, _stream())
+    _check(st, "bns_backward")
+    return dx, dgamma, dbeta
+
+
+def full_bn(x, gamma, beta, eps, y=None, mean=None, invstd=None, workspace=None):
+    """bns_full_bn: ordinary BN forward; returns (y, mean, invstd)."""
+    sh = _shape(x)
+    C = x.shape[1]
+    y = torch.empty_like(x) if y is None else y
+    mean = torch.empty(C, dtype=torch.float32, device=x.device) if mean is None else mean
+    invstd = torch.empty(C, dtype=torch.float32, device=x.device) if invstd is None else invstd
+    ws, wp, wn = _workspace(x, Sampling.full(), workspace)
+    st = load().bns_full_bn(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), _dev(y),
+                            _vec(mean, C), _vec(invstd, C), wp, wn, _stream())
+    _check(st, "bns_full_bn")
+    return y, mean, invstd
+
+
+def selection_mask(x, sampling: Sampling, workspace=None):
+    """bns_debug_selection_mask: uint8 [N,C,H,W]."""
+    sh, sp = _shape(x), sampling._c()
+    mask = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+    ws, wp, wn = _workspace(x, sampling, workspace)
+    _check(load().bns_debug_selection_mask(ctypes.byref(sh), ctypes.byref(sp), mask.data_ptr(), wp, wn, _stream()),
+           "bns_debug_selection_mask")
+    return mask
+
+
+def workspace_status(workspace: torch.Tensor) -> int:
+    flags = ctypes.c_uint32(0)
+    _check(load().bns_workspace_status(workspace.data_ptr(), ctypes.byref(flags), _stream()), "bns_workspace_status")
+    return int(flags.value)
+
+
+# ----------------------------------------------------------------------------- host-buffer step
+def host_arena_bytes(shape, dtype, sampling: Sampling) -> int:
+    N, C, H, W = shape
+    sh = _Shape(N, C, H, W, F32 if dtype == torch.float32 else BF16)
+    sp = sampling._c()
+    return int(load().bns_host_arena_bytes(ctypes.byref(sh), ctypes.byref(sp)))
+
+
+def forward_backward_host(x, dy, gamma, beta, eps, sampling: Sampling, y, dx, mean, invstd, dgamma, dbeta, arena):
+    """bns_forward_backward_host: every tensor argument is a (preferably pinned) HOST tensor except
+    ``arena`` (CUDA uint8 scratch of ``host_arena_bytes``).  Enqueues copies and kernels on the
+    current stream; synchronise before reading the outputs."""
+    for t in (x, dy, gamma, beta, y, dx, mean, invstd, dgamma, dbeta):
+        if t.is_cuda or not t.is_contiguous():
+            raise TypeError("forward_backward_host takes contiguous host tensors")
+    N, C, H, W = x.shape
+    sh = _Shape(N, C, H, W, _dtype_code(x))
+    sp = sampling._c()
+    st = load().bns_forward_backward_host(ctypes.byref(sh), x.data_ptr(), dy.data_ptr(), gamma.data_ptr(),
+                                          beta.data_ptr(), float(eps), ctypes.byref(sp), y.data_ptr(), dx.data_ptr(),
+                                          mean.data_ptr(), invstd.data_ptr(), dgamma.data_ptr(), dbeta.data_ptr(),
+                                          arena.data_ptr(), arena.numel(), _stream())
+    _check(st, "bns_forward_backward_host")
+
+
+# ----------------------------------------------------------------------------- measurement hooks
+def launch_count() -> int:
+    return int(load().bns_launch_count())
+
+
+def launch_count_reset() -> None:
+    load().bns_launch_count_reset()
+
+
+def profile_enable(on: bool) -> None:
+    load().bns_profile_enable(1 if on else 0)
+
+
+def profile_read(kind: int):
+    """(launches, total device milliseconds) of one kernel kind since profiling was enabled."""
+    n, ms = ctypes.c_int(0), ctypes.c_float(0.0)
+    _check(load().bns_profile_read(int(kind), ctypes.byref(n), ctypes.byref(ms)), "bns_profile_read")
+    return int(n.value), float(ms.value)
+
+
+def kernel_name(kind: int) -> str:
+    return load().bns_kernel_name(int(kind)).decode()

@@ -1,0 +1,665 @@
+// Host side of the C ABI declared in include/bns.h: argument validation, launch planning, workspace
+// layout and kernel launches.  Nothing here allocates device memory or synchronises the host (except
+// the two calls that are documented to: bns_workspace_status and bns_profile_read).
+#include "bns.h"
+
+#include <algorithm>
+#include <atomic>
+#include <cstring>
+#include <vector>
+
+#include "bns_kernels.cuh"
+
+namespace {
+
+using namespace bns;
+
+constexpr size_t kAlign = 256;
+constexpr size_t kHeaderBytes = 256;  // status word lives at the start of the workspace
+constexpr int kSmCount = 148;
+
+size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+int elem_bytes(int dtype) { return dtype == BNS_F32 ? 4 : 2; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ------------------------------------------------------------------------------------ measurement hooks
+std::atomic<uint64_t> g_launches{0};
+bool g_profile = false;
+constexpr int kEventPool = 8192;
+struct TimedLaunch {
+    int kind;
+    cudaEvent_t start, stop;
+};
+std::vector<TimedLaunch> g_timed;      // recorded launches since profiling was enabled
+std::vector<cudaEvent_t> g_free_events;
+
+cudaEvent_t take_event() {
+    if (!g_free_events.empty()) {
+        cudaEvent_t e = g_free_events.back();
+        g_free_events.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+struct LaunchScope {
+    cudaStream_t stream;
+    bool timed = false;
+    TimedLaunch rec{};
+    LaunchScope(int kind, cudaStream_t s) : stream(s) {
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (g_profile && static_cast<int>(g_timed.size()) < kEventPool) {
+            rec.kind = kind;
+            rec.start = take_event();
+            rec.stop = take_event();
+            if (rec.start && rec.stop) {
+                timed = true;
+                cudaEventRecord(rec.start, stream);
+            }
+        }
+    }
+    ~LaunchScope() {
+        if (timed) {
+            cudaEventRecord(rec.stop, stream);
+            g_timed.push_back(rec);
+        }
+    }
+};
+
+// ------------------------------------------------------------------------------------ planning
+// How a streaming kernel covers `rows` rows of P positions: vector width, tiles per row, rows per block.
+struct ColPlan {
+    int V = 1;
+    unsigned tiles = 0, TP = 0;
+    int rows = 0, chunk = 0, nchunks = 0, max_slots = 0;
+    unsigned grid() const { return tiles * static_cast<unsigned>(nchunks); }
+    PartialLayout layout() const { return PartialLayout{nchunks, tiles, TP, max_slots}; }
+    size_t partial_count() const { return static_cast<size_t>(nchunks) * tiles * max_slots; }
+};
+
+int g_target_blocks = kSmCount * 32;  // blocks per launch aimed at when splitting the rows into chunks
+int g_min_chunk = 4;                  // but at least this many rows per block
+
+ColPlan plan_col(unsigned P, int HW, int C, int rows, int ebytes) {
+    ColPlan pl;
+    int V = 16 / ebytes;
+    while (V > 1 && P % static_cast<unsigned>(V) != 0) V >>= 1;
+    pl.V = V;
+    pl.TP = static_cast<unsigned>(kThreads) * V;
+    pl.tiles = (P + pl.TP - 1) / pl.TP;
+    pl.rows = rows;
+    long want = (g_target_blocks + static_cast<long>(pl.tiles) - 1) / static_cast<long>(pl.tiles);
+    long nchunks = std::max(1L, std::min<long>(want, std::max(1, rows / g_min_chunk)));
+    pl.chunk = static_cast<int>((rows + nchunks - 1) / nchunks);
+    pl.nchunks = (rows + pl.chunk - 1) / pl.chunk;
+    long slots = (static_cast<long>(pl.TP) + HW - 2) / HW + 1;
+    pl.max_slots = static_cast<int>(std::min<long>(slots, C));
+    return pl;
+}
+
+// Patch kernels: one block per (chunk of samples, channel).
+struct PatchPlan {
+    int chunk = 0, nchunks = 0;
+};
+
+PatchPlan plan_patch(int N, int C, int ph, int pw) {
+    PatchPlan pl;
+    long per_map = static_cast<long>(ph) * pw;
+    long chunk = std::max(1L, std::min<long>(N, 2048 / per_map));
+    // keep enough blocks in flight when C is small
+    while (chunk > 1 && static_cast<long>(C) * ((N + chunk - 1) / chunk) < 4L * kSmCount) chunk = (chunk + 1) / 2;
+    pl.chunk = static_cast<int>(chunk);
+    pl.nchunks = (N + pl.chunk - 1) / pl.chunk;
+    return pl;
+}
+
+struct Problem {
+    int N, C, H, W, HW, dtype;
+    unsigned P;
+    size_t elems;
+    int rule;
+    // resolved sampling
+    int count = 0;                 // BATCH: k; VIRTUAL: nv
+    int begin = 0;                 // BATCH, contiguous ascending list: first index
+    bool contiguous = true;        // BATCH: list is begin .. begin+k-1
+    PatchRule patch{};
+    double s = 0;                  // points per channel that enter the statistics
+    // plans
+    ColPlan main_plan;             // all N rows of x (normalise, backward pass 1, full statistics, full backward)
+    ColPlan stat_plan;             // BATCH: the k sampled rows;  VIRTUAL: the nv rows of xv
+    PatchPlan patch_plan;
+    // workspace layout
+    size_t off_list, off_stats, off_bwd, off_bwd_v, total;
+};
+
+bns_status check_shape(const bns_shape* sh) {
+    if (!sh) return BNS_ERR_NULL;
+    if (sh->N <= 0 || sh->C <= 0 || sh->H <= 0 || sh->W <= 0) return BNS_ERR_SHAPE;
+    if (sh->dtype != BNS_F32 && sh->dtype != BNS_BF16) return BNS_ERR_DTYPE;
+    double P = static_cast<double>(sh->C) * sh->H * sh->W;
+    if (P >= 2147483648.0) return BNS_ERR_SHAPE;              // positions of one sample are indexed with 32 bits
+    if (static_cast<double>(sh->N) * sh->C >= 2147483648.0) return BNS_ERR_SHAPE;
+    return BNS_OK;
+}
+
+// Validates everything that can be validated on the host and fills the plan.
+bns_status make_problem(const bns_shape* sh, const bns_sampling* sp, Problem& pb) {
+    bns_status st = check_shape(sh);
+    if (st != BNS_OK) return st;
+    if (!sp) return BNS_ERR_NULL;
+    pb.N = sh->N;
+    pb.C = sh->C;
+    pb.H = sh->H;
+    pb.W = sh->W;
+    pb.HW = sh->H * sh->W;
+    pb.dtype = sh->dtype;
+    pb.P = static_cast<unsigned>(sh->C) * static_cast<unsigned>(pb.HW);
+    pb.elems = static_cast<size_t>(pb.N) * pb.P;
+    pb.rule = sp->rule;
+    const int eb = elem_bytes(pb.dtype);
+    pb.main_plan = plan_col(pb.P, pb.HW, pb.C, pb.N, eb);
+    pb.stat_plan = pb.main_plan;
+    switch (sp->rule) {
+    case BNS_RULE_FULL:
+        pb.s = static_cast<double>(pb.N) * pb.HW;
+        break;
+    case BNS_RULE_BATCH: {
+        if (sp->k < 1 || sp->k > pb.N) return BNS_ERR_RULE;
+        if (!sp->sample_idx) return BNS_ERR_NULL;
+        std::vector<char> seen(pb.N, 0);
+        pb.contiguous = true;
+        for (int j = 0; j < sp->k; ++j) {
+            int v = sp->sample_idx[j];
+            if (v < 0 || v >= pb.N || seen[v]) return BNS_ERR_INDEX;
+            seen[v] = 1;
+            if (v != sp->sample_idx[0] + j) pb.contiguous = false;
+        }
+        pb.count = sp->k;
+        pb.begin = sp->sample_idx[0];
+        pb.s = static_cast<double>(sp->k) * pb.HW;
+        pb.stat_plan = plan_col(pb.P, pb.HW, pb.C, sp->k, eb);
+        break;
+    }
+    case BNS_RULE_FEATURE: {
+        if (sp->ph < 1 || sp->ph > pb.H || sp->pw < 1 || sp->pw > pb.W) return BNS_ERR_RULE;
+        if (sp->offset_mode < BNS_OFF_SHARED || sp->offset_mode > BNS_OFF_PER_MAP) return BNS_ERR_RULE;
+        if (!sp->offsets) return BNS_ERR_NULL;
+        pb.patch.ph = sp->ph;
+        pb.patch.pw = sp->pw;
+        if (sp->offset_mode == BNS_OFF_SHARED) {
+            int oh = sp->offsets[0], ow = sp->offsets[1];
+            if (oh < 0 || oh > pb.H - sp->ph || ow < 0 || ow > pb.W - sp->pw) return BNS_ERR_INDEX;
+            pb.patch.oh = oh;
+            pb.patch.ow = ow;
+            pb.patch.offsets = nullptr;
+        } else {
+            if (reinterpret_cast<uintptr_t>(sp->offsets) & 7u) return BNS_ERR_ALIGN;
+            pb.patch.offsets = sp->offsets;
+            pb.patch.stride_n = sp->offset_mode == BNS_OFF_PER_SAMPLE ? 1 : pb.C;
+            pb.patch.stride_c = sp->offset_mode == BNS_OFF_PER_SAMPLE ? 0 : 1;
+        }
+        pb.s = static_cast<double>(pb.N) * sp->ph * sp->pw;
+        pb.patch_plan = plan_patch(pb.N, pb.C, sp->ph, sp->pw);
+        break;
+    }
+    case BNS_RULE_VIRTUAL: {
+        if (sp->nv < 1) return BNS_ERR_RULE;
+        if (sp->xv_dtype != BNS_F32 && sp->xv_dtype != BNS_BF16) return BNS_ERR_DTYPE;
+        if (!sp->xv) return BNS_ERR_NULL;
+        if (!aligned16(sp->xv) || !aligned16(sp->yv) || !aligned16(sp->dyv) || !aligned16(sp->dxv)) return BNS_ERR_ALIGN;
+        pb.count = sp->nv;
+        pb.s = static_cast<double>(sp->nv) * pb.HW;
+        pb.stat_plan = plan_col(pb.P, pb.HW, pb.C, sp->nv, elem_bytes(sp->xv_dtype));
+        break;
+    }
+    default:
+        return BNS_ERR_RULE;
+    }
+    // workspace: header | sample list | statistics partials | backward partials (real) | (virtual)
+    size_t off = kHeaderBytes;
+    pb.off_list = off;
+    off += align_up(static_cast<size_t>(pb.N) * sizeof(int));
+    pb.off_stats = off;
+    size_t stat_partials = std::max(pb.main_plan.partial_count(), pb.stat_plan.partial_count());
+    if (sp->rule == BNS_RULE_FEATURE)
+        stat_partials = std::max(stat_partials, static_cast<size_t>(pb.patch_plan.nchunks) * pb.C);
+    off += align_up(stat_partials * sizeof(float4));
+    pb.off_bwd = off;
+    off += align_up(pb.main_plan.partial_count() * sizeof(float2));
+    pb.off_bwd_v = off;
+    if (sp->rule == BNS_RULE_VIRTUAL) off += align_up(pb.stat_plan.partial_count() * sizeof(float2));
+    pb.total = off;
+    return BNS_OK;
+}
+
+bns_status check_workspace(const Problem& pb, const void* ws, size_t bytes) {
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) || bytes < pb.total) return BNS_ERR_WORKSPACE;
+    return BNS_OK;
+}
+
+template <typename T>
+T* ws_at(void* ws, size_t off) {
+    return reinterpret_cast<T*>(static_cast<char*>(ws) + off);
+}
+
+bns_status last_error() { return cudaGetLastError() == cudaSuccess ? BNS_OK : BNS_ERR_CUDA; }
+
+// Copies a non-contiguous sample list into the workspace; returns the device list or NULL.
+bns_status stage_list(const Problem& pb, const bns_sampling* sp, void* ws, cudaStream_t stream, const int** list) {
+    *list = nullptr;
+    if (pb.rule != BNS_RULE_BATCH || pb.contiguous) return BNS_OK;
+    int* dev = ws_at<int>(ws, pb.off_list);
+    if (cudaMemcpyAsync(dev, sp->sample_idx, sizeof(int) * sp->k, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return BNS_ERR_CUDA;
+    *list = dev;
+    return BNS_OK;
+}
+
+bns_status clear_status(const Problem& pb, void* ws, cudaStream_t stream, unsigned** status) {
+    *status = nullptr;
+    if (pb.rule == BNS_RULE_FEATURE && pb.patch.offsets) {
+        if (cudaMemsetAsync(ws, 0, sizeof(unsigned), stream) != cudaSuccess) return BNS_ERR_CUDA;
+        *status = ws_at<unsigned>(ws, 0);
+    }
+    return BNS_OK;
+}
+
+// ------------------------------------------------------------------------------------ typed launches
+template <typename T, int V>
+void launch_col_moments(const ColPlan& pl, const void* x, const int* list,
+                                                                    int begin, int HW, unsigned P, float4* partials,
+                                                                    cudaStream_t s) {
+    LaunchScope scope(BNS_KERNEL_COL_MOMENTS, s);
+    col_moments_kernel<T, V><<<pl.grid(), kThreads, 0, s>>>(static_cast<const typename T::storage*>(x), list, begin,
+                                                            pl.rows, pl.chunk, pl.tiles, HW, P, pl.max_slots, partials);
+}
+
+template <typename T, int V>
+void launch_col_normalize(const ColPlan& pl, const void* x, void* y,
+                                                                      const float* gamma, const float* beta,
+                                                                      const float* mean, const float* invstd, int HW,
+                                                                      unsigned P, cudaStream_t s) {
+    LaunchScope scope(BNS_KERNEL_NORMALIZE, s);
+    col_normalize_kernel<T, V><<<pl.grid(), kThreads, 0, s>>>(static_cast<const typename T::storage*>(x),
+                                                              static_cast<typename T::storage*>(y), gamma, beta, mean,
+                                                              invstd, pl.rows, pl.chunk, pl.tiles, HW, P);
+}
+
+template <typename T, int V>
+void launch_col_bwd_reduce(const ColPlan& pl, const void* x, const void* dy,
+                                                                       void* dx, const float* gamma, const float* mean,
+                                                                       const float* invstd, int HW, unsigned P,
+                                                                       float2* partials, cudaStream_t s) {
+    LaunchScope scope(BNS_KERNEL_BWD_REDUCE, s);
+    using S = typename T::storage;
+    if (dx)
+        col_bwd_reduce_kernel<T, V, true><<<pl.grid(), kThreads, 0, s>>>(
+            static_cast<const S*>(x), static_cast<const S*>(dy), static_cast<S*>(dx), gamma, mean, invstd, pl.rows,
+            pl.chunk, pl.tiles, HW, P, pl.max_slots, partials);
+    else
+        col_bwd_reduce_kernel<T, V, false><<<pl.grid(), kThreads, 0, s>>>(
+            static_cast<const S*>(x), static_cast<const S*>(dy), nullptr, gamma, mean, invstd, pl.rows, pl.chunk,
+            pl.tiles, HW, P, pl.max_slots, partials);
+}
+
+struct BwdParams {
+    const float *gamma, *mean, *invstd, *dgamma, *dbeta;
+    float inv_s;
+};
+
+template <typename T, int V>
+void launch_col_fixup(const ColPlan& pl, const void* x, const void* dy,
+                                                                  void* dx, const BwdParams& bp, const int* list,
+                                                                  int begin, int HW, unsigned P, cudaStream_t s) {
+    LaunchScope scope(BNS_KERNEL_COL_FIXUP, s);
+    using S = typename T::storage;
+    col_fixup_kernel<T, V><<<pl.grid(), kThreads, 0, s>>>(static_cast<const S*>(x), static_cast<const S*>(dy),
+                                                          static_cast<S*>(dx), bp.gamma, bp.mean, bp.invstd, bp.dgamma,
+                                                          bp.dbeta, bp.inv_s, list, begin, pl.rows, pl.chunk, pl.tiles,
+                                                          HW, P);
+}
+
+#define BNS_BY_TYPE_V(dtype, V_, CALL)                   \
+    do {                                                 \
+        if ((dtype) == BNS_F32) {                        \
+            using T = F32;                               \
+            switch (V_) {                                \
+            case 4: { constexpr int V = 4; CALL; } break; \
+            case 2: { constexpr int V = 2; CALL; } break; \
+            default: { constexpr int V = 1; CALL; } break; \
+            }                                            \
+        } else {                                         \
+            using T = BF16;                              \
+            switch (V_) {                                \
+            case 8: { constexpr int V = 8; CALL; } break; \
+            case 4: { constexpr int V = 4; CALL; } break; \
+            case 2: { constexpr int V = 2; CALL; } break; \
+            default: { constexpr int V = 1; CALL; } break; \
+            }                                            \
+        }                                                \
+    } while (0)
+
+void finalize_stats(const float4* partials, PartialLayout L, const Problem& pb, float eps, float* mean, float* invstd,
+                    cudaStream_t s) {
+    LaunchScope scope(BNS_KERNEL_FINALIZE_STATS, s);
+    const int per_block = kThreads / 32;
+    finalize_stats_kernel<<<(pb.C + per_block - 1) / per_block, kThreads, 0, s>>>(
+        partials, L, pb.C, pb.HW, static_cast<float>(pb.s), eps, mean, invstd);
+}
+
+// Statistics of the rule's sampled set into mean / invstd.
+bns_status run_statistics(const Problem& pb, const bns_sampling* sp, const void* x, float eps, float* mean,
+                          float* invstd, void* ws, cudaStream_t stream) {
+    float4* partials = ws_at<float4>(ws, pb.off_stats);
+    if (pb.rule == BNS_RULE_FEATURE) {
+        unsigned* status;
+        bns_status st = clear_status(pb, ws, stream, &status);
+        if (st != BNS_OK) return st;
+        const PatchPlan& pp = pb.patch_plan;
+        const unsigned grid = static_cast<unsigned>(pp.nchunks) * pb.C;
+        {
+            LaunchScope scope(BNS_KERNEL_PATCH_MOMENTS, stream);
+            if (pb.dtype == BNS_F32)
+                patch_moments_kernel<F32><<<grid, kThreads, 0, stream>>>(static_cast<const float*>(x), pb.patch, pb.N,
+                                                                         pb.C, pb.H, pb.W, pp.chunk, partials, status);
+            else
+                patch_moments_kernel<BF16><<<grid, kThreads, 0, stream>>>(static_cast<const unsigned short*>(x),
+                                                                          pb.patch, pb.N, pb.C, pb.H, pb.W, pp.chunk,
+                                                                          partials, status);
+        }
+        PartialLayout L{pp.nchunks, static_cast<unsigned>(pb.C), static_cast<unsigned>(pb.HW), 1};
+        finalize_stats(partials, L, pb, eps, mean, invstd, stream);
+        return last_error();
+    }
+    const int* list = nullptr;
+    bns_status st = stage_list(pb, sp, ws, stream, &list);
+    if (st != BNS_OK) return st;
+    const ColPlan& pl = pb.rule == BNS_RULE_FULL ? pb.main_plan : pb.stat_plan;
+    const void* src = pb.rule == BNS_RULE_VIRTUAL ? sp->xv : x;
+    const int dt = pb.rule == BNS_RULE_VIRTUAL ? sp->xv_dtype : pb.dtype;
+    const int begin = pb.rule == BNS_RULE_BATCH ? pb.begin : 0;
+    BNS_BY_TYPE_V(dt, pl.V, (launch_col_moments<T, V>(pl, src, list, begin, pb.HW, pb.P, partials, stream)));
+    finalize_stats(partials, pl.layout(), pb, eps, mean, invstd, stream);
+    return last_error();
+}
+
+bns_status forward_impl(const Problem& pb, const bns_sampling* sp, const void* x, const float* gamma, const float* beta,
+                        float eps, void* y, float* mean, float* invstd, void* ws, cudaStream_t stream) {
+    bns_status st = run_statistics(pb, sp, x, eps, mean, invstd, ws, stream);
+    if (st != BNS_OK) return st;
+    const ColPlan& pl = pb.main_plan;
+    BNS_BY_TYPE_V(pb.dtype, pl.V,
+                  (launch_col_normalize<T, V>(pl, x, y, gamma, beta, mean, invstd, pb.HW, pb.P, stream)));
+    if (pb.rule == BNS_RULE_VIRTUAL && sp->yv) {
+        const ColPlan& pv = pb.stat_plan;
+        BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
+                      (launch_col_normalize<T, V>(pv, sp->xv, sp->yv, gamma, beta, mean, invstd, pb.HW, pb.P, stream)));
+    }
+    return last_error();
+}
+
+bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* x, const void* dy, const float* gamma,
+                         const float* mean, const float* invstd, void* dx, float* dgamma, float* dbeta, void* ws,
+                         cudaStream_t stream) {
+    const ColPlan& pl = pb.main_plan;
+    float2* partials = ws_at<float2>(ws, pb.off_bwd);
+    float2* partials_v = nullptr;
+    const bool full = pb.rule == BNS_RULE_FULL;
+    // pass 1: the sums of Eq. 5 over every real element; dx = gamma invstd dy everywhere unless every
+    // element is sampled (FULL), where the second pass writes dx anyway.
+    BNS_BY_TYPE_V(pb.dtype, pl.V,
+                  (launch_col_bwd_reduce<T, V>(pl, x, dy, full ? nullptr : dx, gamma, mean, invstd, pb.HW, pb.P,
+                                               partials, stream)));
+    if (pb.rule == BNS_RULE_VIRTUAL && sp->dyv) {
+        const ColPlan& pv = pb.stat_plan;
+        partials_v = ws_at<float2>(ws, pb.off_bwd_v);
+        BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
+                      (launch_col_bwd_reduce<T, V>(pv, sp->xv, sp->dyv, nullptr, gamma, mean, invstd, pb.HW, pb.P,
+                                                   partials_v, stream)));
+    }
+    {
+        LaunchScope scope(BNS_KERNEL_FINALIZE_BWD, stream);
+        const int per_block = kThreads / 32;
+        finalize_bwd_kernel<<<(pb.C + per_block - 1) / per_block, kThreads, 0, stream>>>(
+            partials, pl.layout(), partials_v, pb.stat_plan.layout(), pb.C, pb.HW, invstd, dgamma, dbeta);
+    }
+    // pass 2: the statistics terms, on S only
+    BwdParams bp{gamma, mean, invstd, dgamma, dbeta, static_cast<float>(1.0 / pb.s)};
+    switch (pb.rule) {
+    case BNS_RULE_FULL:
+        BNS_BY_TYPE_V(pb.dtype, pl.V, (launch_col_fixup<T, V>(pl, x, dy, dx, bp, nullptr, 0, pb.HW, pb.P, stream)));
+        break;
+    case BNS_RULE_BATCH: {
+        const int* list = nullptr;
+        bns_status st = stage_list(pb, sp, ws, stream, &list);
+        if (st != BNS_OK) return st;
+        const ColPlan& ps = pb.stat_plan;
+        BNS_BY_TYPE_V(pb.dtype, ps.V, (launch_col_fixup<T, V>(ps, x, dy, dx, bp, list, pb.begin, pb.HW, pb.P, stream)));
+        break;
+    }
+    case BNS_RULE_FEATURE: {
+        unsigned* status;
+        bns_status st = clear_status(pb, ws, stream, &status);
+        if (st != BNS_OK) return st;
+        const PatchPlan& pp = pb.patch_plan;
+        const unsigned grid = static_cast<unsigned>(pp.nchunks) * pb.C;
+        LaunchScope scope(BNS_KERNEL_PATCH_FIXUP, stream);
+        if (pb.dtype == BNS_F32)
+            patch_fixup_kernel<F32><<<grid, kThreads, 0, stream>>>(
+                static_cast<const float*>(x), static_cast<const float*>(dy), static_cast<float*>(dx), gamma, mean,
+                invstd, dgamma, dbeta, bp.inv_s, pb.patch, pb.N, pb.C, pb.H, pb.W, pp.chunk, status);
+        else
+            patch_fixup_kernel<BF16><<<grid, kThreads, 0, stream>>>(
+                static_cast<const unsigned short*>(x), static_cast<const unsigned short*>(dy),
+                static_cast<unsigned short*>(dx), gamma, mean, invstd, dgamma, dbeta, bp.inv_s, pb.patch, pb.N, pb.C,
+                pb.H, pb.W, pp.chunk, status);
+        break;
+    }
+    case BNS_RULE_VIRTUAL:
+        if (sp->dxv) {
+            const ColPlan& pv = pb.stat_plan;
+            BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
+                          (launch_col_fixup<T, V>(pv, sp->xv, sp->dyv, sp->dxv, bp, nullptr, 0, pb.HW, pb.P, stream)));
+        }
+        break;
+    }
+    return last_error();
+}
+
+bns_sampling full_rule() {
+    bns_sampling sp;
+    std::memset(&sp, 0, sizeof(sp));
+    sp.rule = BNS_RULE_FULL;
+    return sp;
+}
+
+}  // namespace
+
+// ======================================================================================== C ABI
+extern "C" {
+
+size_t bns_workspace_bytes(const bns_shape* shape, const bns_sampling* sampling) {
+    Problem pb;
+    if (make_problem(shape, sampling, pb) != BNS_OK) return 0;
+    return pb.total;
+}
+
+bns_status bns_forward(const bns_shape* shape, const void* x, const float* gamma, const float* beta, float eps,
+                       const bns_sampling* sampling, void* y, float* mean, float* invstd, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream) {
+    Problem pb;
+    bns_status st = make_problem(shape, sampling, pb);
+    if (st != BNS_OK) return st;
+    if (!x || !gamma || !beta || !y || !mean || !invstd) return BNS_ERR_NULL;
+    if (!(eps > 0.f)) return BNS_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(y)) return BNS_ERR_ALIGN;
+    st = check_workspace(pb, workspace, workspace_bytes);
+    if (st != BNS_OK) return st;
+    return forward_impl(pb, sampling, x, gamma, beta, eps, y, mean, invstd, workspace,
+                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+bns_status bns_backward(const bns_shape* shape, const void* x, const void* dy, const float* gamma, const float* mean,
+                        const float* invstd, const bns_sampling* sampling, void* dx, float* dgamma, float* dbeta,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    Problem pb;
+    bns_status st = make_problem(shape, sampling, pb);
+    if (st != BNS_OK) return st;
+    if (!x || !dy || !gamma || !mean || !invstd || !dx || !dgamma || !dbeta) return BNS_ERR_NULL;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dx)) return BNS_ERR_ALIGN;
+    st = check_workspace(pb, workspace, workspace_bytes);
+    if (st != BNS_OK) return st;
+    return backward_impl(pb, sampling, x, dy, gamma, mean, invstd, dx, dgamma, dbeta, workspace,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+bns_status bns_full_bn(const bns_shape* shape, const void* x, const float* gamma, const float* beta, float eps, void* y,
+                       float* mean, float* invstd, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    bns_sampling sp = full_rule();
+    return bns_forward(shape, x, gamma, beta, eps, &sp, y, mean, invstd, workspace, workspace_bytes, cuda_stream);
+}
+
+size_t bns_host_arena_bytes(const bns_shape* shape, const bns_sampling* sampling) {
+    Problem pb;
+    if (make_problem(shape, sampling, pb) != BNS_OK) return 0;
+    const size_t tensor = align_up(pb.elems * elem_bytes(pb.dtype));
+    const size_t vec = align_up(static_cast<size_t>(pb.C) * sizeof(float));
+    return 4 * tensor + 6 * vec + align_up(pb.total);
+}
+
+bns_status bns_forward_backward_host(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
+                                     const float* beta, float eps, const bns_sampling* sampling, void* y, void* dx,
+                                     float* mean, float* invstd, float* dgamma, float* dbeta, void* arena,
+                                     size_t arena_bytes, void* cuda_stream) {
+    Problem pb;
+    bns_status st = make_problem(shape, sampling, pb);
+    if (st != BNS_OK) return st;
+    if (!x || !dy || !gamma || !beta || !y || !dx || !mean || !invstd || !dgamma || !dbeta) return BNS_ERR_NULL;
+    if (!(eps > 0.f)) return BNS_ERR_SHAPE;
+    const size_t need = bns_host_arena_bytes(shape, sampling);
+    if (!arena || (reinterpret_cast<uintptr_t>(arena) & (kAlign - 1)) || arena_bytes < need) return BNS_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t tbytes = pb.elems * elem_bytes(pb.dtype);
+    const size_t tensor = align_up(tbytes);
+    const size_t vbytes = static_cast<size_t>(pb.C) * sizeof(float);
+    const size_t vec = align_up(vbytes);
+    char* base = static_cast<char*>(arena);
+    void* d_x = base;
+    void* d_dy = base + tensor;
+    void* d_y = base + 2 * tensor;
+    void* d_dx = base + 3 * tensor;
+    float* d_vec[6];
+    for (int i = 0; i < 6; ++i) d_vec[i] = reinterpret_cast<float*>(base + 4 * tensor + i * vec);
+    void* ws = base + 4 * tensor + 6 * vec;
+    float *d_gamma = d_vec[0], *d_beta = d_vec[1], *d_mean = d_vec[2], *d_invstd = d_vec[3], *d_dgamma = d_vec[4],
+          *d_dbeta = d_vec[5];
+    bool ok = true;
+    ok &= cudaMemcpyAsync(d_x, x, tbytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_gamma, gamma, vbytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_beta, beta, vbytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (!ok) return BNS_ERR_CUDA;
+    st = forward_impl(pb, sampling, d_x, d_gamma, d_beta, eps, d_y, d_mean, d_invstd, ws, stream);
+    if (st != BNS_OK) return st;
+    ok &= cudaMemcpyAsync(y, d_y, tbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_dy, dy, tbytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (!ok) return BNS_ERR_CUDA;
+    st = backward_impl(pb, sampling, d_x, d_dy, d_gamma, d_mean, d_invstd, d_dx, d_dgamma, d_dbeta, ws, stream);
+    if (st != BNS_OK) return st;
+    ok &= cudaMemcpyAsync(dx, d_dx, tbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(mean, d_mean, vbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(invstd, d_invstd, vbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(dgamma, d_dgamma, vbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(dbeta, d_dbeta, vbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    return ok ? BNS_OK : BNS_ERR_CUDA;
+}
+
+bns_status bns_debug_selection_mask(const bns_shape* shape, const bns_sampling* sampling, uint8_t* mask,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    Problem pb;
+    bns_status st = make_problem(shape, sampling, pb);
+    if (st != BNS_OK) return st;
+    if (!mask) return BNS_ERR_NULL;
+    st = check_workspace(pb, workspace, workspace_bytes);
+    if (st != BNS_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int* list = nullptr;
+    st = stage_list(pb, sampling, workspace, stream, &list);
+    if (st != BNS_OK) return st;
+    unsigned* status;
+    st = clear_status(pb, workspace, stream, &status);
+    if (st != BNS_OK) return st;
+    const size_t blocks = std::min<size_t>((pb.elems + kThreads - 1) / kThreads, static_cast<size_t>(kSmCount) * 32);
+    LaunchScope scope(BNS_KERNEL_MASK, stream);
+    selection_mask_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
+        mask, pb.rule, list, pb.begin, pb.count, pb.patch, pb.N, pb.C, pb.H, pb.W, status);
+    return last_error();
+}
+
+bns_status bns_workspace_status(const void* workspace, uint32_t* flags, void* cuda_stream) {
+    if (!workspace || !flags) return BNS_ERR_NULL;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(flags, workspace, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return BNS_ERR_CUDA;
+    return cudaStreamSynchronize(stream) == cudaSuccess ? BNS_OK : BNS_ERR_CUDA;
+}
+
+const char* bns_status_string(bns_status status) {
+    switch (status) {
+    case BNS_OK: return "ok";
+    case BNS_ERR_NULL: return "a required pointer is NULL";
+    case BNS_ERR_SHAPE: return "invalid shape or eps";
+    case BNS_ERR_RULE: return "invalid sampling rule";
+    case BNS_ERR_INDEX: return "sample index or patch offset out of range or repeated";
+    case BNS_ERR_DTYPE: return "unknown element type";
+    case BNS_ERR_ALIGN: return "pointer not sufficiently aligned";
+    case BNS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case BNS_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+uint64_t bns_launch_count(void) { return g_launches.load(); }
+void bns_launch_count_reset(void) { g_launches.store(0); }
+
+void bns_profile_enable(int on) {
+    for (TimedLaunch& t : g_timed) {
+        g_free_events.push_back(t.start);
+        g_free_events.push_back(t.stop);
+    }
+    g_timed.clear();
+    g_profile = on != 0;
+}
+
+bns_status bns_profile_read(int kernel_kind, int* launches, float* total_ms) {
+    if (!launches || !total_ms) return BNS_ERR_NULL;
+    *launches = 0;
+    *total_ms = 0.f;
+    for (const TimedLaunch& t : g_timed) {
+        if (t.kind != kernel_kind) continue;
+        if (cudaEventSynchronize(t.stop) != cudaSuccess) return BNS_ERR_CUDA;
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, t.start, t.stop) != cudaSuccess) return BNS_ERR_CUDA;
+        *launches += 1;
+        *total_ms += ms;
+    }
+    return BNS_OK;
+}
+
+const char* bns_kernel_name(int kernel_kind) {
+    switch (kernel_kind) {
+    case BNS_KERNEL_COL_MOMENTS: return "col_moments_kernel";
+    case BNS_KERNEL_PATCH_MOMENTS: return "patch_moments_kernel";
+    case BNS_KERNEL_FINALIZE_STATS: return "finalize_stats_kernel";
+    case BNS_KERNEL_NORMALIZE: return "col_normalize_kernel";
+    case BNS_KERNEL_BWD_REDUCE: return "col_bwd_reduce_kernel";
+    case BNS_KERNEL_FINALIZE_BWD: return "finalize_bwd_kernel";
+    case BNS_KERNEL_COL_FIXUP: return "col_fixup_kernel";
+    case BNS_KERNEL_PATCH_FIXUP: return "patch_fixup_kernel";
+    case BNS_KERNEL_MASK: return "selection_mask_kernel";
+    }
+    return "unknown";
+}
+
+}  // extern "C"

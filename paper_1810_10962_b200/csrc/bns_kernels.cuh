@@ -1,0 +1,678 @@
+// Device code of the BN-sampling library (sm_100a).
+//
+// Data layout.  A dense NCHW tensor is seen as N rows of P = C*H*W contiguous "positions"; the
+// channel of position p is p / (H*W).  The streaming kernels ("col_*") give every thread V
+// consecutive positions (V elements = up to 16 bytes) and let it walk down the rows n of its chunk:
+// the per-channel parameters of its V positions are looked up once, before the loop, every access
+// is a full-width coalesced vector, and per-channel sums are kept per position in registers, so the
+// inner loop holds no index arithmetic, no shuffles and no shared memory.  Only after the loop are
+// the per-position sums folded into per-channel partials (one block-level pass through shared
+// memory), which a small "finalize" kernel combines across blocks in a fixed order.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace bns {
+
+constexpr int kThreads = 256;  // threads per block of every streaming kernel
+constexpr int kUnroll = 4;     // rows in flight per thread
+
+// ------------------------------------------------------------------------------------ element types
+struct F32 {
+    using storage = float;
+};
+struct BF16 {
+    using storage = unsigned short;
+};
+
+template <typename T>
+__device__ __forceinline__ float to_float(typename T::storage v);
+template <>
+__device__ __forceinline__ float to_float<F32>(float v) {
+    return v;
+}
+template <>
+__device__ __forceinline__ float to_float<BF16>(unsigned short v) {
+    return __uint_as_float(static_cast<unsigned>(v) << 16);
+}
+template <typename T>
+__device__ __forceinline__ typename T::storage from_float(float v);
+template <>
+__device__ __forceinline__ float from_float<F32>(float v) {
+    return v;
+}
+template <>
+__device__ __forceinline__ unsigned short from_float<BF16>(float v) {
+    return __bfloat16_as_ushort(__float2bfloat16_rn(v));  // round to nearest even
+}
+
+template <int BYTES>
+struct RawWord;
+template <>
+struct RawWord<2> {
+    using type = unsigned short;
+};
+template <>
+struct RawWord<4> {
+    using type = unsigned;
+};
+template <>
+struct RawWord<8> {
+    using type = uint2;
+};
+template <>
+struct RawWord<16> {
+    using type = uint4;
+};
+
+// V consecutive elements moved as one machine word of 2..16 bytes.
+template <typename T, int V>
+struct Vec {
+    using S = typename T::storage;
+    using raw_t = typename RawWord<sizeof(S) * V>::type;
+    raw_t raw;
+    __device__ __forceinline__ void load(const S* p) { raw = *reinterpret_cast<const raw_t*>(p); }
+    __device__ __forceinline__ void store(S* p) const { *reinterpret_cast<raw_t*>(p) = raw; }
+    __device__ __forceinline__ float get(int j) const { return to_float<T>(reinterpret_cast<const S*>(&raw)[j]); }
+    __device__ __forceinline__ void set(int j, float v) { reinterpret_cast<S*>(&raw)[j] = from_float<T>(v); }
+};
+
+// Channels of the V positions p .. p+V-1 (HW may be smaller than V).
+template <int V>
+__device__ __forceinline__ void position_channels(unsigned p, int HW, int (&c)[V]) {
+    int c0 = static_cast<int>(p / static_cast<unsigned>(HW));
+    int r = static_cast<int>(p - static_cast<unsigned>(c0) * static_cast<unsigned>(HW));
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        c[j] = c0;
+        if (++r == HW) {
+            r = 0;
+            ++c0;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------ moments
+// (count, mean, sum of squared deviations) of a set; merge() is the pairwise update of Chan et al.
+struct Moments {
+    float cnt, mean, m2;
+};
+
+__device__ __forceinline__ Moments merge(Moments a, Moments b) {
+    float n = a.cnt + b.cnt;
+    if (n == 0.f) return a;
+    float d = b.mean - a.mean;
+    float f = b.cnt / n;
+    Moments r;
+    r.cnt = n;
+    r.mean = a.mean + d * f;
+    r.m2 = a.m2 + b.m2 + d * d * a.cnt * f;
+    return r;
+}
+
+__device__ __forceinline__ Moments shuffle_down(Moments m, int delta) {
+    Moments r;
+    r.cnt = __shfl_down_sync(0xffffffffu, m.cnt, delta);
+    r.mean = __shfl_down_sync(0xffffffffu, m.mean, delta);
+    r.m2 = __shfl_down_sync(0xffffffffu, m.m2, delta);
+    return r;
+}
+
+__device__ __forceinline__ Moments warp_merge(Moments m) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) m = merge(m, shuffle_down(m, d));
+    return m;  // complete in lane 0
+}
+
+// Moments of one position from sums shifted by a pivot K that is itself one of the values:
+// sum1 = sum(x-K), sum2 = sum((x-K)^2) over cnt values.
+__device__ __forceinline__ Moments from_shifted_sums(float cnt, float K, float sum1, float sum2) {
+    Moments m;
+    m.cnt = cnt;
+    if (cnt == 0.f) {
+        m.mean = 0.f;
+        m.m2 = 0.f;
+        return m;
+    }
+    float d = sum1 / cnt;
+    m.mean = K + d;
+    m.m2 = fmaxf(sum2 - sum1 * d, 0.f);
+    return m;
+}
+
+// Where a block's tile of positions [p0, p0+TP) meets the channels: slot j is channel c_first + j.
+struct TileChannels {
+    unsigned p0, pend;
+    int c_first, nslots;
+    __device__ __forceinline__ TileChannels(unsigned tile, unsigned TP, unsigned P, int HW) {
+        p0 = tile * TP;
+        pend = min(p0 + TP, P);
+        c_first = static_cast<int>(p0 / static_cast<unsigned>(HW));
+        nslots = static_cast<int>((pend - 1) / static_cast<unsigned>(HW)) - c_first + 1;
+    }
+    // positions of slot j, relative to p0
+    __device__ __forceinline__ void range(int slot, int HW, unsigned& lo, unsigned& hi) const {
+        unsigned cb = static_cast<unsigned>(c_first + slot) * static_cast<unsigned>(HW);
+        lo = max(cb, p0) - p0;
+        hi = min(cb + static_cast<unsigned>(HW), pend) - p0;
+    }
+};
+
+// ------------------------------------------------------------------------------------ statistics over whole samples
+// Partial moments of x[list, :] per (row chunk, tile, channel slot).  `list` (device) holds the
+// sample indices or is NULL for the contiguous range begin .. begin+count-1.
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+col_moments_kernel(const typename T::storage* __restrict__ x, const int* __restrict__ list, int begin, int count,
+                   int chunk, unsigned tiles, int HW, unsigned P, int max_slots, float4* __restrict__ partials) {
+    constexpr unsigned TP = kThreads * V;
+    __shared__ float s_mean[TP];
+    __shared__ float s_m2[TP];
+    const unsigned tile = blockIdx.x % tiles;
+    const unsigned ck = blockIdx.x / tiles;
+    const unsigned p = (tile * kThreads + threadIdx.x) * V;
+    const int i0 = ck * chunk, i1 = min(count, i0 + chunk);
+    const float cnt = static_cast<float>(i1 - i0);
+    float K[V], s1[V], s2[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) K[j] = s1[j] = s2[j] = 0.f;
+    if (p < P) {
+        const typename T::storage* xp = x + p;
+        {
+            int n = list ? list[i0] : begin + i0;
+            Vec<T, V> v;
+            v.load(xp + static_cast<size_t>(n) * P);
+#pragma unroll
+            for (int j = 0; j < V; ++j) K[j] = v.get(j);
+        }
+        int i = i0 + 1;
+        for (; i + kUnroll <= i1; i += kUnroll) {
+            Vec<T, V> v[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                int n = list ? list[i + u] : begin + i + u;
+                v[u].load(xp + static_cast<size_t>(n) * P);
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+#pragma unroll
+                for (int j = 0; j < V; ++j) {
+                    float d = v[u].get(j) - K[j];
+                    s1[j] += d;
+                    s2[j] = fmaf(d, d, s2[j]);
+                }
+        }
+        for (; i < i1; ++i) {
+            int n = list ? list[i] : begin + i;
+            Vec<T, V> v;
+            v.load(xp + static_cast<size_t>(n) * P);
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                float d = v.get(j) - K[j];
+                s1[j] += d;
+                s2[j] = fmaf(d, d, s2[j]);
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        Moments m = from_shifted_sums(cnt, K[j], s1[j], s2[j]);
+        s_mean[threadIdx.x * V + j] = m.mean;
+        s_m2[threadIdx.x * V + j] = m.m2;
+    }
+    __syncthreads();
+    const TileChannels tc(tile, TP, P, HW);
+    float4* out = partials + (static_cast<size_t>(ck) * tiles + tile) * max_slots;
+    if (HW >= 32) {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int slot = warp; slot < tc.nslots; slot += kThreads / 32) {
+            unsigned lo, hi;
+            tc.range(slot, HW, lo, hi);
+            Moments acc = {0.f, 0.f, 0.f};
+            for (unsigned q = lo + lane; q < hi; q += 32) acc = merge(acc, Moments{cnt, s_mean[q], s_m2[q]});
+            acc = warp_merge(acc);
+            if (lane == 0) out[slot] = make_float4(acc.cnt, acc.mean, acc.m2, 0.f);
+        }
+    } else {
+        for (int slot = threadIdx.x; slot < tc.nslots; slot += kThreads) {
+            unsigned lo, hi;
+            tc.range(slot, HW, lo, hi);
+            Moments acc = {0.f, 0.f, 0.f};
+            for (unsigned q = lo; q < hi; ++q) acc = merge(acc, Moments{cnt, s_mean[q], s_m2[q]});
+            out[slot] = make_float4(acc.cnt, acc.mean, acc.m2, 0.f);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------ statistics over patches
+// Patch location of map (n, c): one pair for the layer, one per sample or one per map.  Pairs read
+// from device memory are clamped into range; an out-of-range pair raises a flag in `status`.
+struct PatchRule {
+    int ph, pw;
+    int oh, ow;          // SHARED location (validated on the host)
+    const int* offsets;  // device pairs or NULL for SHARED
+    int stride_n, stride_c;
+};
+
+__device__ __forceinline__ void patch_origin(const PatchRule& r, int n, int c, int H, int W, unsigned* status, int& oh,
+                                             int& ow) {
+    if (!r.offsets) {
+        oh = r.oh;
+        ow = r.ow;
+        return;
+    }
+    size_t e = static_cast<size_t>(n) * r.stride_n + static_cast<size_t>(c) * r.stride_c;
+    int2 o = reinterpret_cast<const int2*>(r.offsets)[e];
+    oh = min(max(o.x, 0), H - r.ph);
+    ow = min(max(o.y, 0), W - r.pw);
+    if ((oh != o.x || ow != o.y) && status) atomicOr(status, 1u);
+}
+
+// One block per (sample chunk, channel): threads stride over the patch elements of the chunk's maps.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+patch_moments_kernel(const typename T::storage* __restrict__ x, PatchRule rule, int N, int C, int H, int W, int chunk,
+                     float4* __restrict__ partials, unsigned* status) {
+    __shared__ Moments s_warp[kThreads / 32];
+    const int c = blockIdx.x % C;
+    const int ck = blockIdx.x / C;
+    const int n0 = ck * chunk, n1 = min(N, n0 + chunk);
+    const int PP = rule.ph * rule.pw;
+    const int total = (n1 - n0) * PP;
+    const size_t HW = static_cast<size_t>(H) * W;
+    float K = 0.f, s1 = 0.f, s2 = 0.f, cnt = 0.f;
+    for (int q = threadIdx.x; q < total; q += kThreads) {
+        int nl = q / PP, e = q - nl * PP;
+        int r = e / rule.pw, col = e - r * rule.pw;
+        int n = n0 + nl, oh, ow;
+        patch_origin(rule, n, c, H, W, status, oh, ow);
+        float v = to_float<T>(x[(static_cast<size_t>(n) * C + c) * HW + static_cast<size_t>(oh + r) * W + ow + col]);
+        if (cnt == 0.f) K = v;
+        float d = v - K;
+        s1 += d;
+        s2 = fmaf(d, d, s2);
+        cnt += 1.f;
+    }
+    Moments m = warp_merge(from_shifted_sums(cnt, K, s1, s2));
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        Moments acc = s_warp[0];
+        for (int w = 1; w < kThreads / 32; ++w) acc = merge(acc, s_warp[w]);
+        partials[static_cast<size_t>(ck) * C + c] = make_float4(acc.cnt, acc.mean, acc.m2, 0.f);
+    }
+}
+
+// ------------------------------------------------------------------------------------ finalize
+// How the partials of one pass are indexed: partial[(chunk*tiles + tile)*max_slots + slot], where
+// tile t covers positions [t*TP, (t+1)*TP) of a row and slot = channel - first channel of the tile.
+// The per-(chunk, channel) layout of the patch kernels is the case TP = HW, tiles = C, max_slots = 1.
+struct PartialLayout {
+    int nchunks;
+    unsigned tiles, TP;
+    int max_slots;
+};
+
+// One warp per channel merges its partial moments in a fixed order and writes mean and invstd.
+__global__ void __launch_bounds__(kThreads)
+finalize_stats_kernel(const float4* __restrict__ partials, PartialLayout L, int C, int HW, float s, float eps,
+                      float* __restrict__ mean, float* __restrict__ invstd) {
+    const int c = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (c >= C) return;
+    const unsigned pb = static_cast<unsigned>(c) * HW;
+    const unsigned t_lo = pb / L.TP, t_hi = (pb + HW - 1) / L.TP;
+    const int nt = static_cast<int>(t_hi - t_lo + 1);
+    const int entries = L.nchunks * nt;
+    Moments acc = {0.f, 0.f, 0.f};
+    for (int e = lane; e < entries; e += 32) {
+        int ck = e / nt;
+        unsigned t = t_lo + static_cast<unsigned>(e - ck * nt);
+        int slot = c - static_cast<int>((t * L.TP) / static_cast<unsigned>(HW));
+        float4 v = partials[(static_cast<size_t>(ck) * L.tiles + t) * L.max_slots + slot];
+        acc = merge(acc, Moments{v.x, v.y, v.z});
+    }
+    acc = warp_merge(acc);
+    if (lane == 0) {
+        float var = acc.m2 / s;
+        mean[c] = acc.mean;
+        invstd[c] = 1.0f / sqrtf(var + eps);
+    }
+}
+
+// One warp per channel adds its partial (sum dy, sum dy (x - mean)) pairs in a fixed order, from the
+// real tensor and, when present, from the virtual samples.
+__global__ void __launch_bounds__(kThreads)
+finalize_bwd_kernel(const float2* __restrict__ partials, PartialLayout L, const float2* __restrict__ partials_v,
+                    PartialLayout Lv, int C, int HW, const float* __restrict__ invstd, float* __restrict__ dgamma,
+                    float* __restrict__ dbeta) {
+    const int c = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (c >= C) return;
+    const unsigned pb = static_cast<unsigned>(c) * HW;
+    float sum_dy = 0.f, sum_dyxc = 0.f;
+    for (int pass = 0; pass < 2; ++pass) {
+        const float2* src = pass ? partials_v : partials;
+        if (!src) continue;
+        const PartialLayout& Q = pass ? Lv : L;
+        const unsigned t_lo = pb / Q.TP, t_hi = (pb + HW - 1) / Q.TP;
+        const int nt = static_cast<int>(t_hi - t_lo + 1);
+        const int entries = Q.nchunks * nt;
+        for (int e = lane; e < entries; e += 32) {
+            int ck = e / nt;
+            unsigned t = t_lo + static_cast<unsigned>(e - ck * nt);
+            int slot = c - static_cast<int>((t * Q.TP) / static_cast<unsigned>(HW));
+            float2 v = src[(static_cast<size_t>(ck) * Q.tiles + t) * Q.max_slots + slot];
+            sum_dy += v.x;
+            sum_dyxc += v.y;
+        }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        sum_dy += __shfl_down_sync(0xffffffffu, sum_dy, d);
+        sum_dyxc += __shfl_down_sync(0xffffffffu, sum_dyxc, d);
+    }
+    if (lane == 0) {
+        dbeta[c] = sum_dy;
+        dgamma[c] = sum_dyxc * invstd[c];
+    }
+}
+
+// ------------------------------------------------------------------------------------ normalise + affine
+// y = a_c x + b_c with a_c = gamma_c invstd_c and b_c = beta_c - mean_c a_c, over rows [n0, n1).
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::storage* __restrict__ y,
+                     const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
+                     const float* __restrict__ invstd, int rows, int chunk, unsigned tiles, int HW, unsigned P) {
+    const unsigned tile = blockIdx.x % tiles;
+    const unsigned ck = blockIdx.x / tiles;
+    const unsigned p = (tile * kThreads + threadIdx.x) * V;
+    if (p >= P) return;
+    float a[V], b[V];
+    {
+        int c[V];
+        position_channels<V>(p, HW, c);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            a[j] = gamma[c[j]] * invstd[c[j]];
+            b[j] = fmaf(-mean[c[j]], a[j], beta[c[j]]);
+        }
+    }
+    const int n0 = ck * chunk, n1 = min(rows, n0 + chunk);
+    const typename T::storage* xp = x + static_cast<size_t>(n0) * P + p;
+    typename T::storage* yp = y + static_cast<size_t>(n0) * P + p;
+    int n = n0;
+    for (; n + kUnroll <= n1; n += kUnroll) {
+        Vec<T, V> v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) v[u].load(xp + static_cast<size_t>(u) * P);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+#pragma unroll
+            for (int j = 0; j < V; ++j) v[u].set(j, fmaf(a[j], v[u].get(j), b[j]));
+            v[u].store(yp + static_cast<size_t>(u) * P);
+        }
+        xp += static_cast<size_t>(kUnroll) * P;
+        yp += static_cast<size_t>(kUnroll) * P;
+    }
+    for (; n < n1; ++n) {
+        Vec<T, V> v;
+        v.load(xp);
+#pragma unroll
+        for (int j = 0; j < V; ++j) v.set(j, fmaf(a[j], v.get(j), b[j]));
+        v.store(yp);
+        xp += P;
+        yp += P;
+    }
+}
+
+// ------------------------------------------------------------------------------------ backward, pass 1
+// Streams dy and x once: per channel partial sums of dy and dy (x - mean) and, if WRITE_DX, the
+// gradient of every element without the statistics terms, dx = gamma invstd dy (lower branch of Eq. 6).
+template <typename T, int V, bool WRITE_DX>
+__global__ void __launch_bounds__(kThreads)
+col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
+                      typename T::storage* __restrict__ dx, const float* __restrict__ gamma,
+                      const float* __restrict__ mean, const float* __restrict__ invstd, int rows, int chunk,
+                      unsigned tiles, int HW, unsigned P, int max_slots, float2* __restrict__ partials) {
+    constexpr unsigned TP = kThreads * V;
+    __shared__ float s_dy[TP];
+    __shared__ float s_dyxc[TP];
+    const unsigned tile = blockIdx.x % tiles;
+    const unsigned ck = blockIdx.x / tiles;
+    const unsigned p = (tile * kThreads + threadIdx.x) * V;
+    float acc_dy[V], acc_dyxc[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc_dy[j] = acc_dyxc[j] = 0.f;
+    if (p < P) {
+        float a[V], mu[V];
+        {
+            int c[V];
+            position_channels<V>(p, HW, c);
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                mu[j] = mean[c[j]];
+                a[j] = WRITE_DX ? gamma[c[j]] * invstd[c[j]] : 0.f;
+            }
+        }
+        const int n0 = ck * chunk, n1 = min(rows, n0 + chunk);
+        const size_t base = static_cast<size_t>(n0) * P + p;
+        const typename T::storage* xp = x + base;
+        const typename T::storage* gp = dy + base;
+        typename T::storage* op = WRITE_DX ? dx + base : nullptr;
+        int n = n0;
+        for (; n + kUnroll <= n1; n += kUnroll) {
+            Vec<T, V> vx[kUnroll], vg[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                vx[u].load(xp + static_cast<size_t>(u) * P);
+                vg[u].load(gp + static_cast<size_t>(u) * P);
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+#pragma unroll
+                for (int j = 0; j < V; ++j) {
+                    float g = vg[u].get(j);
+                    acc_dy[j] += g;
+                    acc_dyxc[j] = fmaf(g, vx[u].get(j) - mu[j], acc_dyxc[j]);
+                    if (WRITE_DX) vg[u].set(j, a[j] * g);
+                }
+                if (WRITE_DX) vg[u].store(op + static_cast<size_t>(u) * P);
+            }
+            xp += static_cast<size_t>(kUnroll) * P;
+            gp += static_cast<size_t>(kUnroll) * P;
+            if (WRITE_DX) op += static_cast<size_t>(kUnroll) * P;
+        }
+        for (; n < n1; ++n) {
+            Vec<T, V> vx, vg;
+            vx.load(xp);
+            vg.load(gp);
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                float g = vg.get(j);
+                acc_dy[j] += g;
+                acc_dyxc[j] = fmaf(g, vx.get(j) - mu[j], acc_dyxc[j]);
+                if (WRITE_DX) vg.set(j, a[j] * g);
+            }
+            if (WRITE_DX) {
+                vg.store(op);
+                op += P;
+            }
+            xp += P;
+            gp += P;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        s_dy[threadIdx.x * V + j] = acc_dy[j];
+        s_dyxc[threadIdx.x * V + j] = acc_dyxc[j];
+    }
+    __syncthreads();
+    const TileChannels tc(tile, TP, P, HW);
+    float2* out = partials + (static_cast<size_t>(ck) * tiles + tile) * max_slots;
+    if (HW >= 32) {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int slot = warp; slot < tc.nslots; slot += kThreads / 32) {
+            unsigned lo, hi;
+            tc.range(slot, HW, lo, hi);
+            float sa = 0.f, sb = 0.f;
+            for (unsigned q = lo + lane; q < hi; q += 32) {
+                sa += s_dy[q];
+                sb += s_dyxc[q];
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                sa += __shfl_down_sync(0xffffffffu, sa, d);
+                sb += __shfl_down_sync(0xffffffffu, sb, d);
+            }
+            if (lane == 0) out[slot] = make_float2(sa, sb);
+        }
+    } else {
+        for (int slot = threadIdx.x; slot < tc.nslots; slot += kThreads) {
+            unsigned lo, hi;
+            tc.range(slot, HW, lo, hi);
+            float sa = 0.f, sb = 0.f;
+            for (unsigned q = lo; q < hi; ++q) {
+                sa += s_dy[q];
+                sb += s_dyxc[q];
+            }
+            out[slot] = make_float2(sa, sb);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------ backward, statistics terms
+// Per-channel coefficients of the full gradient of a sampled element (upper branch of Eq. 6):
+//   dx = a dy - A - Q (x - mean),  a = gamma invstd,  A = a dbeta / s,  Q = a invstd dgamma / s.
+struct FixCoef {
+    float a, A, Q, mu;
+};
+
+__device__ __forceinline__ FixCoef fix_coef(int c, const float* gamma, const float* mean, const float* invstd,
+                                            const float* dgamma, const float* dbeta, float inv_s) {
+    FixCoef k;
+    float is = invstd[c];
+    k.a = gamma[c] * is;
+    k.A = k.a * dbeta[c] * inv_s;
+    k.Q = k.a * is * dgamma[c] * inv_s;
+    k.mu = mean[c];
+    return k;
+}
+
+// Rows given by `list` (or begin .. begin+count-1): dx = a dy - A - Q (x - mean); dy == NULL reads as zeros.
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
+                 typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
+                 const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
+                 float inv_s, const int* __restrict__ list, int begin, int count, int chunk, unsigned tiles, int HW,
+                 unsigned P) {
+    const unsigned tile = blockIdx.x % tiles;
+    const unsigned ck = blockIdx.x / tiles;
+    const unsigned p = (tile * kThreads + threadIdx.x) * V;
+    if (p >= P) return;
+    FixCoef k[V];
+    {
+        int c[V];
+        position_channels<V>(p, HW, c);
+#pragma unroll
+        for (int j = 0; j < V; ++j) k[j] = fix_coef(c[j], gamma, mean, invstd, dgamma, dbeta, inv_s);
+    }
+    const int i0 = ck * chunk, i1 = min(count, i0 + chunk);
+    int i = i0;
+    for (; i + 2 <= i1; i += 2) {
+        Vec<T, V> vx[2], vg[2];
+        size_t off[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            int n = list ? list[i + u] : begin + i + u;
+            off[u] = static_cast<size_t>(n) * P + p;
+            vx[u].load(x + off[u]);
+            if (dy) vg[u].load(dy + off[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                float g = dy ? vg[u].get(j) : 0.f;
+                vg[u].set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (vx[u].get(j) - k[j].mu));
+            }
+            vg[u].store(dx + off[u]);
+        }
+    }
+    for (; i < i1; ++i) {
+        int n = list ? list[i] : begin + i;
+        size_t off = static_cast<size_t>(n) * P + p;
+        Vec<T, V> vx, vg;
+        vx.load(x + off);
+        if (dy) vg.load(dy + off);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            float g = dy ? vg.get(j) : 0.f;
+            vg.set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (vx.get(j) - k[j].mu));
+        }
+        vg.store(dx + off);
+    }
+}
+
+// The same for the patch elements of the chunk's maps of one channel.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
+                   typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
+                   const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
+                   float inv_s, PatchRule rule, int N, int C, int H, int W, int chunk, unsigned* status) {
+    const int c = blockIdx.x % C;
+    const int ck = blockIdx.x / C;
+    const int n0 = ck * chunk, n1 = min(N, n0 + chunk);
+    const int PP = rule.ph * rule.pw;
+    const int total = (n1 - n0) * PP;
+    const size_t HW = static_cast<size_t>(H) * W;
+    const FixCoef k = fix_coef(c, gamma, mean, invstd, dgamma, dbeta, inv_s);
+    for (int q = threadIdx.x; q < total; q += kThreads) {
+        int nl = q / PP, e = q - nl * PP;
+        int r = e / rule.pw, col = e - r * rule.pw;
+        int n = n0 + nl, oh, ow;
+        patch_origin(rule, n, c, H, W, status, oh, ow);
+        size_t at = (static_cast<size_t>(n) * C + c) * HW + static_cast<size_t>(oh + r) * W + ow + col;
+        float g = to_float<T>(dy[at]);
+        float xv = to_float<T>(x[at]);
+        dx[at] = from_float<T>(fmaf(k.a, g, -k.A) - k.Q * (xv - k.mu));
+    }
+}
+
+// ------------------------------------------------------------------------------------ selection mask (test aid)
+__global__ void __launch_bounds__(kThreads)
+selection_mask_kernel(uint8_t* __restrict__ mask, int rule, const int* __restrict__ list, int begin, int count,
+                      PatchRule patch, int N, int C, int H, int W, unsigned* status) {
+    const size_t total = static_cast<size_t>(N) * C * H * W;
+    for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < total;
+         i += static_cast<size_t>(gridDim.x) * kThreads) {
+        int w = static_cast<int>(i % W);
+        size_t t = i / W;
+        int h = static_cast<int>(t % H);
+        t /= H;
+        int c = static_cast<int>(t % C);
+        int n = static_cast<int>(t / C);
+        uint8_t in = 0;
+        if (rule == 0) {
+            in = 1;
+        } else if (rule == 1) {
+            if (list) {
+                for (int j = 0; j < count; ++j) in |= (list[j] == n);
+            } else {
+                in = n >= begin && n < begin + count;
+            }
+        } else if (rule == 2) {
+            int oh, ow;
+            patch_origin(patch, n, c, H, W, status, oh, ow);
+            in = h >= oh && h < oh + patch.ph && w >= ow && w < ow + patch.pw;
+        }
+        mask[i] = in;
+    }
+}
+
+}  // namespace bns

@@ -1,0 +1,93 @@
+"""CPU-side checks of the C ABI: the library loads without a GPU, exports every symbol the header
+declares, and rejects bad arguments on the host before anything is launched."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_1810_10962_b200 import bns
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "bns.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(bns_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = bns.load()
+    names = declared_symbols()
+    assert {"bns_forward", "bns_backward", "bns_full_bn", "bns_workspace_bytes"} <= set(names)
+    for name in names:
+        assert hasattr(lib, name), name
+    assert set(names) == set(bns.EXPORTS)
+
+
+def test_status_strings():
+    assert bns.status_string(0) == "ok"
+    for code in range(-8, 0):
+        assert bns.status_string(code) not in ("ok", "unknown status")
+
+
+def _call_forward(shape, sp, x=0x1000, gamma=0x2000, beta=0x3000, y=0x4000, mean=0x5000, invstd=0x6000, eps=1e-5,
+                  ws=0x10000, ws_bytes=1 << 30):
+    """Fake, never dereferenced device addresses: every case below must be refused on the host."""
+    lib = bns.load()
+    sh = bns._Shape(*shape)
+    return lib.bns_forward(ctypes.byref(sh), x, gamma, beta, eps, ctypes.byref(sp), y, mean, invstd, ws, ws_bytes, None)
+
+
+def test_forward_rejects_bad_arguments_before_launching():
+    idx = np.array([0, 1], np.int32)
+    ok = bns.Sampling.batch(idx)._c()
+    shape = (8, 16, 8, 8, bns.F32)
+    assert _call_forward((0, 16, 8, 8, 0), ok) == -2                       # N = 0
+    assert _call_forward((8, 16, 8, 8, 7), ok) == -5                       # dtype
+    assert _call_forward((8, 1 << 15, 1 << 10, 1 << 10, 0), ok) == -2      # C*H*W overflows 31 bits
+    assert _call_forward(shape, ok, x=0) == -1                             # null x
+    assert _call_forward(shape, ok, x=0x1004) == -6                        # misaligned x
+    assert _call_forward(shape, ok, eps=0.0) == -2
+    assert _call_forward(shape, ok, ws=0) == -7
+    assert _call_forward(shape, ok, ws=0x10010) == -7                      # workspace not 256-aligned
+    assert _call_forward(shape, ok, ws_bytes=16) == -7
+    for bad in ([0, 0], [0, 8], [-1, 2]):                                  # repeated / out of range
+        sp = bns.Sampling.batch(np.array(bad, np.int32))._c()
+        assert _call_forward(shape, sp) == -4
+    sp = bns.Sampling.batch(np.arange(9, dtype=np.int32))._c()             # k > N
+    assert _call_forward(shape, sp) == -3
+    sp = bns.Sampling.feature(9, 2, np.array([0, 0]))._c()                 # patch taller than the map
+    assert _call_forward(shape, sp) == -3
+    sp = bns.Sampling.feature(3, 3, np.array([6, 0]))._c()                 # patch leaves the map
+    assert _call_forward(shape, sp) == -4
+    sp = bns.Sampling.feature(3, 3, np.array([0, -1]))._c()
+    assert _call_forward(shape, sp) == -4
+    sp = bns._Sampling()
+    sp.rule = 9
+    assert _call_forward(shape, sp) == -3
+    sp = bns._Sampling()
+    sp.rule, sp.nv = bns.RULE_VIRTUAL, 0
+    assert _call_forward(shape, sp) == -3
+    sp.nv = 2                                                              # xv missing
+    assert _call_forward(shape, sp) == -1
+
+
+def test_workspace_bytes_is_zero_for_invalid_and_stable_for_valid():
+    lib = bns.load()
+    sh = bns._Shape(256, 64, 56, 56, bns.F32)
+    sp = bns.Sampling.batch(np.arange(32, dtype=np.int32))._c()
+    a = lib.bns_workspace_bytes(ctypes.byref(sh), ctypes.byref(sp))
+    assert a > 0 and a == lib.bns_workspace_bytes(ctypes.byref(sh), ctypes.byref(sp)) and a % 256 == 0
+    bad = bns._Shape(256, 64, 56, -1, bns.F32)
+    assert lib.bns_workspace_bytes(ctypes.byref(bad), ctypes.byref(sp)) == 0
+
+
+def test_binding_refuses_cpu_tensors():
+    import torch
+    x = torch.zeros(2, 3, 4, 4)
+    with pytest.raises(TypeError):
+        bns.forward(x, torch.ones(3), torch.zeros(3), 1e-5, bns.Sampling.full(),
+                    workspace=torch.empty(1 << 20, dtype=torch.uint8))

@@ -1,0 +1,182 @@
+"""GPU parity: the C ABI against the CPU oracle, element by element, on the five benchmark
+configurations and on the edge cases."""
+import numpy as np
+import pytest
+
+import bns_inputs as I
+import oracle as O
+from helpers import Case, compare, gpu_sampling, make_case, run_gpu, _to_device
+
+pytestmark = pytest.mark.gpu
+
+
+# ----------------------------------------------------------------------------- config 1: tiny
+@pytest.mark.parametrize("rule,kw", [
+    ("batch", dict(k=2, contiguous=False)),
+    ("batch", dict(k=2, contiguous=True)),
+    ("feature", dict(ph=3, pw=3, offset_mode=0)),
+    ("feature", dict(ph=2, pw=5, offset_mode=1)),
+    ("feature", dict(ph=4, pw=1, offset_mode=2)),
+    ("virtual", dict(nv=2)),
+    ("virtual", dict(nv=1, with_dyv=False)),
+    ("full", dict()),
+])
+def test_config1_tiny(rule, kw):
+    case = make_case(8, 16, 8, 8, rule, seed=1811, generator="tiny", **kw)
+    compare(case, run_gpu(case))
+
+
+# ----------------------------------------------------------------------------- config 2: CIFAR sweep
+@pytest.mark.parametrize("C,H", I.cifar_resnet_layers())
+@pytest.mark.parametrize("mode", [0, 2])
+def test_config2_cifar_feature_sampling(C, H, mode):
+    case = make_case(128, C, H, H, "feature", seed=1812, ph=4, pw=4, offset_mode=mode)
+    compare(case, run_gpu(case))
+
+
+# ----------------------------------------------------------------------------- config 3: ResNet-18 stage 1, full size
+@pytest.mark.parametrize("rule,kw", [
+    ("batch", dict(k=32, contiguous=True)),
+    ("feature", dict(ph=8, pw=8, offset_mode=0)),
+    ("full", dict()),
+])
+def test_config3_resnet18_stage1_full_size(rule, kw):
+    case = make_case(256, 64, 56, 56, rule, seed=1813, **kw)
+    g = run_gpu(case)
+    compare(case, g, channels=[0, 1, 31, 32, 63])       # the oracle checks these channels completely
+
+
+# ----------------------------------------------------------------------------- config 4: VDN, bf16 activations
+def test_config4_vdn_bf16():
+    case = make_case(256, 128, 28, 28, "virtual", seed=1814, dtype="bf16", nv=2, xv_dtype="f32", with_dyv=False)
+    compare(case, run_gpu(case), channels=[0, 5, 64, 127])
+
+
+# ----------------------------------------------------------------------------- config 5: ResNet-50 sweep, bf16
+def _distinct_resnet50():
+    return sorted(set(I.resnet50_bn_layers()), key=lambda t: (-t[1], t[0]))
+
+
+@pytest.mark.parametrize("C,H", _distinct_resnet50())
+def test_config5_resnet50_layers_full_size(C, H):
+    p = max(1, H // 8)
+    case = make_case(256, C, H, H, "feature", seed=1815, dtype="bf16", ph=p, pw=p, offset_mode=0)
+    compare(case, run_gpu(case), channels=[0, C // 2 + 1, C - 1])
+
+
+# ----------------------------------------------------------------------------- edge cases
+EDGE = [
+    # odd everything: one element per vector
+    dict(N=3, C=3, H=5, W=7, rule="feature", ph=5, pw=7),                  # patch = whole map
+    dict(N=3, C=3, H=5, W=7, rule="feature", ph=1, pw=1, offset_mode=2),   # one point per map
+    dict(N=5, C=7, H=3, W=3, rule="batch", k=1),
+    dict(N=5, C=7, H=3, W=3, rule="batch", k=5, contiguous=False),         # ratio 1
+    dict(N=1, C=4, H=6, W=6, rule="full"),
+    dict(N=2, C=130, H=1, W=1, rule="batch", k=1),                         # fully connected layer: HW = 1
+    dict(N=64, C=40, H=1, W=1, rule="full"),
+    dict(N=9, C=12, H=2, W=2, rule="virtual", nv=3),                       # HW smaller than a vector
+    dict(N=4, C=6, H=7, W=7, rule="feature", ph=3, pw=2, offset_mode=1, dtype="bf16"),   # P*2 % 16 != 0
+    dict(N=4, C=8, H=7, W=7, rule="batch", k=3, contiguous=False, dtype="bf16"),         # 98-byte maps
+    dict(N=6, C=16, H=14, W=14, rule="full", dtype="bf16"),
+    dict(N=6, C=16, H=14, W=14, rule="virtual", nv=2, dtype="bf16", xv_dtype="bf16"),
+    dict(N=70, C=5, H=33, W=31, rule="batch", k=9),                        # several row chunks, ragged tile tail
+    dict(N=37, C=300, H=4, W=4, rule="feature", ph=2, pw=3, offset_mode=2),
+]
+
+
+@pytest.mark.parametrize("spec", EDGE, ids=lambda s: "-".join(f"{k}{v}" for k, v in s.items()))
+def test_edge_cases(spec):
+    spec = dict(spec)
+    dims = [spec.pop(k) for k in ("N", "C", "H", "W")]
+    rule = spec.pop("rule")
+    case = make_case(*dims, rule, seed=77, generator="tiny", **spec)
+    compare(case, run_gpu(case))
+
+
+def test_patch_at_every_border():
+    N, C, H, W = 4, 5, 9, 11
+    for oh, ow in [(0, 0), (0, W - 4), (H - 3, 0), (H - 3, W - 4)]:
+        case = make_case(N, C, H, W, "feature", seed=78, generator="tiny", ph=3, pw=4)
+        case.offsets = np.array([[oh, ow]], np.int32)
+        compare(case, run_gpu(case))
+
+
+def test_full_bn_entry_point_equals_full_rule():
+    case = make_case(16, 24, 10, 10, "full", seed=79)
+    a, b = run_gpu(case, use_full_bn_entry=True), run_gpu(case)
+    for key in ("y", "mean", "invstd", "dx", "dgamma", "dbeta"):
+        assert np.array_equal(getattr(a, key), getattr(b, key)), key
+    compare(case, a)
+
+
+def test_ratio_one_matches_full_bn_on_gpu():
+    """Batch Sampling with every sample and Feature Sampling with the whole map are ordinary BN."""
+    full = make_case(12, 10, 6, 6, "full", seed=80)
+    gf = run_gpu(full)
+    bs = make_case(12, 10, 6, 6, "batch", seed=80, k=12)
+    fs = make_case(12, 10, 6, 6, "feature", seed=80, ph=6, pw=6)
+    for case in (bs, fs):
+        g = run_gpu(case)
+        compare(case, g)
+        np.testing.assert_allclose(g.y, gf.y, rtol=1e-5, atol=1e-5)
+        np.testing.assert_allclose(g.dx, gf.dx, rtol=1e-4, atol=1e-5)
+
+
+# ----------------------------------------------------------------------------- selection is bit-exact
+@pytest.mark.parametrize("rule,kw", [
+    ("batch", dict(k=5, contiguous=False)), ("batch", dict(k=4, contiguous=True)),
+    ("feature", dict(ph=3, pw=2, offset_mode=0)), ("feature", dict(ph=3, pw=2, offset_mode=1)),
+    ("feature", dict(ph=1, pw=4, offset_mode=2)), ("virtual", dict()), ("full", dict()),
+])
+def test_selection_mask_bit_exact(rule, kw):
+    from paper_1810_10962_b200 import bns
+    case = make_case(11, 6, 7, 9, rule, seed=81, generator="tiny", **kw)
+    x = _to_device(case.x, "f32")
+    mask = bns.selection_mask(x, gpu_sampling(case)).cpu().numpy()
+    assert np.array_equal(mask, O.selection_mask(11, 6, 7, 9, case.oracle_sampling()))
+
+
+def test_selection_sentinel_through_the_statistics():
+    """x = 1 exactly on S, 0 elsewhere -> the GPU statistics must be mean 1, var 0 (invstd eps^-1/2)."""
+    for rule, kw in [("batch", dict(k=3, contiguous=False)), ("feature", dict(ph=2, pw=3, offset_mode=2))]:
+        case = make_case(10, 6, 8, 8, rule, seed=82, generator="tiny", **kw)
+        case.x = O.selection_mask(10, 6, 8, 8, case.oracle_sampling()).astype(np.float32)
+        g = run_gpu(case)
+        assert np.array_equal(g.mean, np.ones(6, np.float32))
+        np.testing.assert_allclose(g.invstd, np.float32(1e-5) ** -0.5, rtol=1e-6)
+
+
+# ----------------------------------------------------------------------------- determinism
+@pytest.mark.parametrize("rule,kw", [("batch", dict(k=8)), ("feature", dict(ph=4, pw=4)), ("full", dict())])
+def test_runs_are_bit_identical(rule, kw):
+    import torch
+    case = make_case(64, 32, 28, 28, rule, seed=83, **kw)
+    a, b = run_gpu(case), run_gpu(case)
+    for key in a.raw:
+        assert torch.equal(a.raw[key], b.raw[key]), key
+
+
+# ----------------------------------------------------------------------------- device-resident offsets are checked
+def test_bad_device_offsets_raise_flag_and_stay_in_bounds():
+    import torch
+    from paper_1810_10962_b200 import bns
+    case = make_case(4, 3, 6, 6, "feature", seed=84, generator="tiny", ph=2, pw=2, offset_mode=1)
+    x = _to_device(case.x, "f32")
+    gamma, beta = torch.from_numpy(case.gamma).cuda(), torch.from_numpy(case.beta).cuda()
+    good = torch.from_numpy(case.offsets).cuda()
+    sp = bns.Sampling.feature(2, 2, good, bns.OFF_PER_SAMPLE)
+    ws = bns.new_workspace(x, sp)
+    bns.forward(x, gamma, beta, 1e-5, sp, workspace=ws)
+    assert bns.workspace_status(ws) == 0
+    bad = good.clone()
+    bad[1, 0] = 99
+    bad[2, 1] = -3
+    sp_bad = bns.Sampling.feature(2, 2, bad, bns.OFF_PER_SAMPLE)
+    y, mean, invstd = bns.forward(x, gamma, beta, 1e-5, sp_bad, workspace=ws)
+    assert bns.workspace_status(ws) & bns.FLAG_BAD_OFFSET
+    # clamped into range: same as the nearest valid offsets
+    clamped = case.offsets.copy()
+    clamped[1, 0], clamped[2, 1] = 4, 0
+    case.offsets = clamped
+    f = O.forward(case.x, case.gamma, case.beta, 1e-5, case.oracle_sampling())
+    np.testing.assert_allclose(mean.cpu().numpy(), f.mean, atol=1e-5)
