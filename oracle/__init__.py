@@ -126,6 +126,11 @@ def _check_offsets(sp: Sampling, N, C, H, W):
         assert sp.nv >= 1
 
 
+def threads() -> int:
+    """Host threads the oracle's channel loop uses."""
+    return int(_library().oracle_threads())
+
+
 def sample_count(N, H, W, sp: Sampling) -> int:
     c, _keep = sp._c()
     return int(_library().oracle_sample_count(N, H, W, ctypes.byref(c)))

@@ -237,6 +237,14 @@ void oracle_backward(int N, int C, int H, int W, const float *x, const float *xv
     }
 }
 
+/* Host threads the channel loops run on (1 without OpenMP). */
+#ifdef _OPENMP
+#include <omp.h>
+int oracle_threads(void) { return omp_get_max_threads(); }
+#else
+int oracle_threads(void) { return 1; }
+#endif
+
 /* Appendix C.1: with an adder tree the depth falls from log(m) to log(s), a ratio of log_s(m). */
 double oracle_adder_tree_depth_ratio(int N, int H, int W, const oracle_sampling *sp)
 {
