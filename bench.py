@@ -285,6 +285,9 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     bns.load()
+    for item in args.tune:
+        name, value = item.split("=")
+        bns.set_tuning(name, int(value))
     layers, seeds = selected_layers(args)
     hosts = [host_inputs(l, s) for l, s in zip(layers, seeds)]
     bytes_per_tensor_set = sum(4 * l.elems * l.ebytes for l in layers)
@@ -375,7 +378,8 @@ def run_ours(args):
             "config": {"workload": args.workload + (f" (only {args.only})" if args.only else ""),
                        "layers": [f"{l.name}:{l.N}x{l.C}x{l.H}x{l.W}:{l.dtype}:x{l.count}" for l in layers],
                        "step": "forward+backward of every layer", "algorithmic_bytes_per_step": step_bytes,
-                       "cache": f"inputs larger than L2; {sets} buffer sets rotated", "replicas": world},
+                       "cache": f"inputs larger than L2; {sets} buffer sets rotated", "replicas": world,
+                       "tuning": args.tune},
             "frac_of_hbm_peak": round(value / world / peak, 4), "hbm_peak_gbs": peak, "hbm_peak_source": peak_source,
             "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
             "clocks": clocks_plain, "e2e": e2e, "gpu_launches": int(launches),
@@ -523,6 +527,8 @@ def main():
     ap.add_argument("--workload", default="resnet18_stage1",
                     choices=["resnet18_stage1", "cifar", "vdn", "resnet50", "tiny"])
     ap.add_argument("--only", default=None, help="comma-separated layer names: run just these layers of the workload")
+    ap.add_argument("--tune", action="append", default=[], metavar="NAME=VALUE",
+                    help="launch-shape knob of the library (bns_set_tuning), e.g. --tune pdl=0")
     ap.add_argument("--no-full-bn", dest="full_bn", action="store_false", help="skip the full-BN comparison")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--e2e-steps", type=int, default=5)

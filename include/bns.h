@@ -18,8 +18,8 @@
  *    that nothing was enqueued.  No exception crosses this boundary.
  *  - Results are a deterministic function of the inputs: no floating-point atomics are used and
  *    every cross-block combine runs in a fixed order, so two runs give identical bits.
- *  - `workspace` is scratch of at least bns_workspace_bytes() bytes, 256-byte aligned.  Calls that
- *    overlap in time on the GPU need distinct workspaces.
+ *  - `workspace` is scratch of at least bns_workspace_bytes() bytes, 256-byte aligned; its contents
+ *    need no initialisation.  Calls that overlap in time on the GPU need distinct workspaces.
  */
 #ifndef BNS_H
 #define BNS_H
@@ -180,6 +180,13 @@ void bns_launch_count_reset(void);
 void bns_profile_enable(int on);
 bns_status bns_profile_read(int kernel_kind, int* launches, float* total_ms);
 const char* bns_kernel_name(int kernel_kind);
+
+/* Launch-shape knobs (process-wide; change them only while no call is in flight, and recompute
+ * bns_workspace_bytes afterwards).  "target_blocks" / "min_chunk": blocks per launch and least rows
+ * per block of the streaming kernels; "stat_target_blocks" / "stat_min_chunk": the same for the
+ * statistics kernels; "pdl": 0/1 programmatic dependent launch.  Returns BNS_OK,
+ * BNS_ERR_RULE for an unknown name or BNS_ERR_SHAPE for a value < 1. */
+int bns_set_tuning(const char* name, int value);
 
 #ifdef __cplusplus
 }

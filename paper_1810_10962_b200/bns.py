@@ -31,6 +31,7 @@ EXPORTS = [
     "bns_workspace_bytes", "bns_forward", "bns_backward", "bns_full_bn", "bns_host_arena_bytes",
     "bns_forward_backward_host", "bns_debug_selection_mask", "bns_workspace_status", "bns_status_string",
     "bns_launch_count", "bns_launch_count_reset", "bns_profile_enable", "bns_profile_read", "bns_kernel_name",
+    "bns_set_tuning",
 ]
 
 
@@ -101,6 +102,8 @@ def load():
     lib.bns_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float)]
     lib.bns_kernel_name.restype = ctypes.c_char_p
     lib.bns_kernel_name.argtypes = [ctypes.c_int]
+    lib.bns_set_tuning.restype = ctypes.c_int
+    lib.bns_set_tuning.argtypes = [ctypes.c_char_p, ctypes.c_int]
     _lib = lib
     return lib
 
@@ -220,6 +223,7 @@ def workspace_bytes(x: torch.Tensor, sampling: Sampling) -> int:
 
 
 def new_workspace(x: torch.Tensor, sampling: Sampling) -> torch.Tensor:
+    """Allocate a workspace for this shape and rule."""
     return torch.empty(workspace_bytes(x, sampling), dtype=torch.uint8, device=x.device)
 
 
@@ -333,6 +337,11 @@ def profile_read(kind: int):
     n, ms = ctypes.c_int(0), ctypes.c_float(0.0)
     _check(load().bns_profile_read(int(kind), ctypes.byref(n), ctypes.byref(ms)), "bns_profile_read")
     return int(n.value), float(ms.value)
+
+
+def set_tuning(name: str, value: int) -> None:
+    """bns_set_tuning: launch-shape knobs (see include/bns.h)."""
+    _check(load().bns_set_tuning(name.encode(), int(value)), f"bns_set_tuning({name})")
 
 
 def kernel_name(kind: int) -> str:

@@ -79,10 +79,14 @@ struct ColPlan {
     size_t partial_count() const { return static_cast<size_t>(nchunks) * tiles * max_slots; }
 };
 
-int g_target_blocks = kSmCount * 32;  // blocks per launch aimed at when splitting the rows into chunks
-int g_min_chunk = 4;                  // but at least this many rows per block
+int g_target_blocks = kSmCount * 8;       // streaming kernels: blocks per launch aimed at when splitting the rows
+int g_min_chunk = 4;                      // ... but at least this many rows per block
+int g_stat_target_blocks = kSmCount * 8;  // short statistics kernels: one wave of blocks, all loads in flight
+int g_stat_min_chunk = 1;
 
-ColPlan plan_col(unsigned P, int HW, int C, int rows, int ebytes) {
+ColPlan plan_col(unsigned P, int HW, int C, int rows, int ebytes, bool statistics = false) {
+    const int target_blocks = statistics ? g_stat_target_blocks : g_target_blocks;
+    const int min_chunk = statistics ? g_stat_min_chunk : g_min_chunk;
     ColPlan pl;
     int V = 16 / ebytes;
     while (V > 1 && P % static_cast<unsigned>(V) != 0) V >>= 1;
@@ -90,8 +94,9 @@ ColPlan plan_col(unsigned P, int HW, int C, int rows, int ebytes) {
     pl.TP = static_cast<unsigned>(kThreads) * V;
     pl.tiles = (P + pl.TP - 1) / pl.TP;
     pl.rows = rows;
-    long want = (g_target_blocks + static_cast<long>(pl.tiles) - 1) / static_cast<long>(pl.tiles);
-    long nchunks = std::max(1L, std::min<long>(want, std::max(1, rows / g_min_chunk)));
+    // as many row chunks as keep the grid within the target (one wave of resident blocks)
+    long want = target_blocks / static_cast<long>(pl.tiles);
+    long nchunks = std::max(1L, std::min<long>(want, std::max(1, rows / min_chunk)));
     pl.chunk = static_cast<int>((rows + nchunks - 1) / nchunks);
     pl.nchunks = (rows + pl.chunk - 1) / pl.chunk;
     long slots = (static_cast<long>(pl.TP) + HW - 2) / HW + 1;
@@ -99,19 +104,25 @@ ColPlan plan_col(unsigned P, int HW, int C, int rows, int ebytes) {
     return pl;
 }
 
-// Patch kernels: one block per (chunk of samples, channel).
+// Patch kernels: a sample row has C*ph*pw compact positions, 256 per block.
 struct PatchPlan {
-    int chunk = 0, nchunks = 0;
+    unsigned tiles = 0;
+    int chunk = 0, nchunks = 0, max_slots = 0;
+    unsigned grid() const { return tiles * static_cast<unsigned>(nchunks); }
+    PartialLayout layout() const { return PartialLayout{nchunks, tiles, static_cast<unsigned>(kThreads), max_slots}; }
+    size_t partial_count() const { return static_cast<size_t>(nchunks) * tiles * max_slots; }
 };
 
 PatchPlan plan_patch(int N, int C, int ph, int pw) {
     PatchPlan pl;
-    long per_map = static_cast<long>(ph) * pw;
-    long chunk = std::max(1L, std::min<long>(N, 2048 / per_map));
-    // keep enough blocks in flight when C is small
-    while (chunk > 1 && static_cast<long>(C) * ((N + chunk - 1) / chunk) < 4L * kSmCount) chunk = (chunk + 1) / 2;
-    pl.chunk = static_cast<int>(chunk);
+    const long PP = static_cast<long>(ph) * pw;
+    const long Pc = static_cast<long>(C) * PP;
+    pl.tiles = static_cast<unsigned>((Pc + kThreads - 1) / kThreads);
+    long want = g_stat_target_blocks / static_cast<long>(pl.tiles);
+    long nchunks = std::max(1L, std::min<long>(want, std::max(1, N / 4)));
+    pl.chunk = static_cast<int>((N + nchunks - 1) / nchunks);
     pl.nchunks = (N + pl.chunk - 1) / pl.chunk;
+    pl.max_slots = static_cast<int>(std::min<long>((kThreads + PP - 2) / PP + 1, C));
     return pl;
 }
 
@@ -179,7 +190,7 @@ bns_status make_problem(const bns_shape* sh, const bns_sampling* sp, Problem& pb
         pb.count = sp->k;
         pb.begin = sp->sample_idx[0];
         pb.s = static_cast<double>(sp->k) * pb.HW;
-        pb.stat_plan = plan_col(pb.P, pb.HW, pb.C, sp->k, eb);
+        pb.stat_plan = plan_col(pb.P, pb.HW, pb.C, sp->k, eb, true);
         break;
     }
     case BNS_RULE_FEATURE: {
@@ -211,7 +222,7 @@ bns_status make_problem(const bns_shape* sh, const bns_sampling* sp, Problem& pb
         if (!aligned16(sp->xv) || !aligned16(sp->yv) || !aligned16(sp->dyv) || !aligned16(sp->dxv)) return BNS_ERR_ALIGN;
         pb.count = sp->nv;
         pb.s = static_cast<double>(sp->nv) * pb.HW;
-        pb.stat_plan = plan_col(pb.P, pb.HW, pb.C, sp->nv, elem_bytes(sp->xv_dtype));
+        pb.stat_plan = plan_col(pb.P, pb.HW, pb.C, sp->nv, elem_bytes(sp->xv_dtype), true);
         break;
     }
     default:
@@ -224,7 +235,7 @@ bns_status make_problem(const bns_shape* sh, const bns_sampling* sp, Problem& pb
     pb.off_stats = off;
     size_t stat_partials = std::max(pb.main_plan.partial_count(), pb.stat_plan.partial_count());
     if (sp->rule == BNS_RULE_FEATURE)
-        stat_partials = std::max(stat_partials, static_cast<size_t>(pb.patch_plan.nchunks) * pb.C);
+        stat_partials = std::max(stat_partials, pb.patch_plan.partial_count());
     off += align_up(stat_partials * sizeof(float4));
     pb.off_bwd = off;
     off += align_up(pb.main_plan.partial_count() * sizeof(float2));
@@ -266,59 +277,23 @@ bns_status clear_status(const Problem& pb, void* ws, cudaStream_t stream, unsign
     return BNS_OK;
 }
 
-// ------------------------------------------------------------------------------------ typed launches
-template <typename T, int V>
-void launch_col_moments(const ColPlan& pl, const void* x, const int* list,
-                                                                    int begin, int HW, unsigned P, float4* partials,
-                                                                    cudaStream_t s) {
-    LaunchScope scope(BNS_KERNEL_COL_MOMENTS, s);
-    col_moments_kernel<T, V><<<pl.grid(), kThreads, 0, s>>>(static_cast<const typename T::storage*>(x), list, begin,
-                                                            pl.rows, pl.chunk, pl.tiles, HW, P, pl.max_slots, partials);
-}
+// ------------------------------------------------------------------------------------ launches
+bool g_pdl = true;    // ask for programmatic dependent launch (blocks may be scheduled while the previous kernel drains)
 
-template <typename T, int V>
-void launch_col_normalize(const ColPlan& pl, const void* x, void* y,
-                                                                      const float* gamma, const float* beta,
-                                                                      const float* mean, const float* invstd, int HW,
-                                                                      unsigned P, cudaStream_t s) {
-    LaunchScope scope(BNS_KERNEL_NORMALIZE, s);
-    col_normalize_kernel<T, V><<<pl.grid(), kThreads, 0, s>>>(static_cast<const typename T::storage*>(x),
-                                                              static_cast<typename T::storage*>(y), gamma, beta, mean,
-                                                              invstd, pl.rows, pl.chunk, pl.tiles, HW, P);
-}
-
-template <typename T, int V>
-void launch_col_bwd_reduce(const ColPlan& pl, const void* x, const void* dy,
-                                                                       void* dx, const float* gamma, const float* mean,
-                                                                       const float* invstd, int HW, unsigned P,
-                                                                       float2* partials, cudaStream_t s) {
-    LaunchScope scope(BNS_KERNEL_BWD_REDUCE, s);
-    using S = typename T::storage;
-    if (dx)
-        col_bwd_reduce_kernel<T, V, true><<<pl.grid(), kThreads, 0, s>>>(
-            static_cast<const S*>(x), static_cast<const S*>(dy), static_cast<S*>(dx), gamma, mean, invstd, pl.rows,
-            pl.chunk, pl.tiles, HW, P, pl.max_slots, partials);
-    else
-        col_bwd_reduce_kernel<T, V, false><<<pl.grid(), kThreads, 0, s>>>(
-            static_cast<const S*>(x), static_cast<const S*>(dy), nullptr, gamma, mean, invstd, pl.rows, pl.chunk,
-            pl.tiles, HW, P, pl.max_slots, partials);
-}
-
-struct BwdParams {
-    const float *gamma, *mean, *invstd, *dgamma, *dbeta;
-    float inv_s;
-};
-
-template <typename T, int V>
-void launch_col_fixup(const ColPlan& pl, const void* x, const void* dy,
-                                                                  void* dx, const BwdParams& bp, const int* list,
-                                                                  int begin, int HW, unsigned P, cudaStream_t s) {
-    LaunchScope scope(BNS_KERNEL_COL_FIXUP, s);
-    using S = typename T::storage;
-    col_fixup_kernel<T, V><<<pl.grid(), kThreads, 0, s>>>(static_cast<const S*>(x), static_cast<const S*>(dy),
-                                                          static_cast<S*>(dx), bp.gamma, bp.mean, bp.invstd, bp.dgamma,
-                                                          bp.dbeta, bp.inv_s, list, begin, pl.rows, pl.chunk, pl.tiles,
-                                                          HW, P);
+template <typename... KArgs, typename... Args>
+void launch(int kind, void (*kernel)(KArgs...), unsigned grid, cudaStream_t s, Args&&... args) {
+    LaunchScope scope(kind, s);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 #define BNS_BY_TYPE_V(dtype, V_, CALL)                   \
@@ -341,47 +316,56 @@ void launch_col_fixup(const ColPlan& pl, const void* x, const void* dy,
         }                                                \
     } while (0)
 
-void finalize_stats(const float4* partials, PartialLayout L, const Problem& pb, float eps, float* mean, float* invstd,
-                    cudaStream_t s) {
-    LaunchScope scope(BNS_KERNEL_FINALIZE_STATS, s);
-    const int per_block = kThreads / 32;
-    finalize_stats_kernel<<<(pb.C + per_block - 1) / per_block, kThreads, 0, s>>>(
-        partials, L, pb.C, pb.HW, static_cast<float>(pb.s), eps, mean, invstd);
+#define BNS_BY_TYPE(dtype, CALL)   \
+    do {                           \
+        if ((dtype) == BNS_F32) {  \
+            using T = F32;         \
+            CALL;                  \
+        } else {                   \
+            using T = BF16;        \
+            CALL;                  \
+        }                          \
+    } while (0)
+
+template <typename T>
+const typename T::storage* in(const void* p) {
+    return static_cast<const typename T::storage*>(p);
+}
+template <typename T>
+typename T::storage* out(void* p) {
+    return static_cast<typename T::storage*>(p);
 }
 
-// Statistics of the rule's sampled set into mean / invstd.
+unsigned warp_per_channel_grid(int C) { return static_cast<unsigned>((C + kThreads / 32 - 1) / (kThreads / 32)); }
+
+// Statistics of the rule's sampled set into mean / invstd: partial moments, then one warp per channel.
 bns_status run_statistics(const Problem& pb, const bns_sampling* sp, const void* x, float eps, float* mean,
                           float* invstd, void* ws, cudaStream_t stream) {
-    float4* partials = ws_at<float4>(ws, pb.off_stats);
+    StatsSink sink{ws_at<float4>(ws, pb.off_stats), PartialLayout{}, static_cast<float>(1.0 / pb.s), eps, mean, invstd};
+    int span = pb.HW;  // positions per channel in the producer's position space
     if (pb.rule == BNS_RULE_FEATURE) {
         unsigned* status;
         bns_status st = clear_status(pb, ws, stream, &status);
         if (st != BNS_OK) return st;
         const PatchPlan& pp = pb.patch_plan;
-        const unsigned grid = static_cast<unsigned>(pp.nchunks) * pb.C;
-        {
-            LaunchScope scope(BNS_KERNEL_PATCH_MOMENTS, stream);
-            if (pb.dtype == BNS_F32)
-                patch_moments_kernel<F32><<<grid, kThreads, 0, stream>>>(static_cast<const float*>(x), pb.patch, pb.N,
-                                                                         pb.C, pb.H, pb.W, pp.chunk, partials, status);
-            else
-                patch_moments_kernel<BF16><<<grid, kThreads, 0, stream>>>(static_cast<const unsigned short*>(x),
-                                                                          pb.patch, pb.N, pb.C, pb.H, pb.W, pp.chunk,
-                                                                          partials, status);
-        }
-        PartialLayout L{pp.nchunks, static_cast<unsigned>(pb.C), static_cast<unsigned>(pb.HW), 1};
-        finalize_stats(partials, L, pb, eps, mean, invstd, stream);
-        return last_error();
+        sink.L = pp.layout();
+        span = pb.patch.ph * pb.patch.pw;
+        BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_MOMENTS, patch_moments_kernel<T>, pp.grid(), stream, in<T>(x),
+                                      pb.patch, pb.N, pb.C, pb.H, pb.W, pp.chunk, pp.tiles, sink, status)));
+    } else {
+        const int* list = nullptr;
+        bns_status st = stage_list(pb, sp, ws, stream, &list);
+        if (st != BNS_OK) return st;
+        const ColPlan& pl = pb.rule == BNS_RULE_FULL ? pb.main_plan : pb.stat_plan;
+        const void* data = pb.rule == BNS_RULE_VIRTUAL ? sp->xv : x;
+        const int dt = pb.rule == BNS_RULE_VIRTUAL ? sp->xv_dtype : pb.dtype;
+        const int begin = pb.rule == BNS_RULE_BATCH ? pb.begin : 0;
+        sink.L = pl.layout();
+        BNS_BY_TYPE_V(dt, pl.V,
+                      (launch(BNS_KERNEL_COL_MOMENTS, col_moments_kernel<T, V>, pl.grid(), stream, in<T>(data), list, begin,
+                              pl.rows, pl.chunk, pl.tiles, pb.HW, pb.P, sink)));
     }
-    const int* list = nullptr;
-    bns_status st = stage_list(pb, sp, ws, stream, &list);
-    if (st != BNS_OK) return st;
-    const ColPlan& pl = pb.rule == BNS_RULE_FULL ? pb.main_plan : pb.stat_plan;
-    const void* src = pb.rule == BNS_RULE_VIRTUAL ? sp->xv : x;
-    const int dt = pb.rule == BNS_RULE_VIRTUAL ? sp->xv_dtype : pb.dtype;
-    const int begin = pb.rule == BNS_RULE_BATCH ? pb.begin : 0;
-    BNS_BY_TYPE_V(dt, pl.V, (launch_col_moments<T, V>(pl, src, list, begin, pb.HW, pb.P, partials, stream)));
-    finalize_stats(partials, pl.layout(), pb, eps, mean, invstd, stream);
+    launch(BNS_KERNEL_FINALIZE_STATS, finalize_stats_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, span);
     return last_error();
 }
 
@@ -391,11 +375,13 @@ bns_status forward_impl(const Problem& pb, const bns_sampling* sp, const void* x
     if (st != BNS_OK) return st;
     const ColPlan& pl = pb.main_plan;
     BNS_BY_TYPE_V(pb.dtype, pl.V,
-                  (launch_col_normalize<T, V>(pl, x, y, gamma, beta, mean, invstd, pb.HW, pb.P, stream)));
+                  (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pl.grid(), stream, in<T>(x), out<T>(y), gamma,
+                          beta, mean, invstd, pl.rows, pl.chunk, pl.tiles, pb.HW, pb.P)));
     if (pb.rule == BNS_RULE_VIRTUAL && sp->yv) {
         const ColPlan& pv = pb.stat_plan;
         BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
-                      (launch_col_normalize<T, V>(pv, sp->xv, sp->yv, gamma, beta, mean, invstd, pb.HW, pb.P, stream)));
+                      (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pv.grid(), stream, in<T>(sp->xv),
+                              out<T>(sp->yv), gamma, beta, mean, invstd, pv.rows, pv.chunk, pv.tiles, pb.HW, pb.P)));
     }
     return last_error();
 }
@@ -404,39 +390,46 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
                          const float* mean, const float* invstd, void* dx, float* dgamma, float* dbeta, void* ws,
                          cudaStream_t stream) {
     const ColPlan& pl = pb.main_plan;
-    float2* partials = ws_at<float2>(ws, pb.off_bwd);
-    float2* partials_v = nullptr;
+    const ColPlan& pv = pb.stat_plan;
     const bool full = pb.rule == BNS_RULE_FULL;
+    const bool virtual_grads = pb.rule == BNS_RULE_VIRTUAL && sp->dyv;
+    GradSink sink{ws_at<float2>(ws, pb.off_bwd), pl.layout(), virtual_grads ? ws_at<float2>(ws, pb.off_bwd_v) : nullptr,
+                  pv.layout(), invstd, dgamma, dbeta};
     // pass 1: the sums of Eq. 5 over every real element; dx = gamma invstd dy everywhere unless every
     // element is sampled (FULL), where the second pass writes dx anyway.
-    BNS_BY_TYPE_V(pb.dtype, pl.V,
-                  (launch_col_bwd_reduce<T, V>(pl, x, dy, full ? nullptr : dx, gamma, mean, invstd, pb.HW, pb.P,
-                                               partials, stream)));
-    if (pb.rule == BNS_RULE_VIRTUAL && sp->dyv) {
-        const ColPlan& pv = pb.stat_plan;
-        partials_v = ws_at<float2>(ws, pb.off_bwd_v);
+    if (full)
+        BNS_BY_TYPE_V(pb.dtype, pl.V,
+                      (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, false>, pl.grid(), stream, in<T>(x),
+                              in<T>(dy), out<T>(nullptr), gamma, mean, invstd, pl.rows, pl.chunk, pl.tiles, pb.HW, pb.P,
+                              false, sink)));
+    else
+        BNS_BY_TYPE_V(pb.dtype, pl.V,
+                      (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, true>, pl.grid(), stream, in<T>(x),
+                              in<T>(dy), out<T>(dx), gamma, mean, invstd, pl.rows, pl.chunk, pl.tiles, pb.HW, pb.P, false,
+                              sink)));
+    if (virtual_grads)
         BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
-                      (launch_col_bwd_reduce<T, V>(pv, sp->xv, sp->dyv, nullptr, gamma, mean, invstd, pb.HW, pb.P,
-                                                   partials_v, stream)));
-    }
-    {
-        LaunchScope scope(BNS_KERNEL_FINALIZE_BWD, stream);
-        const int per_block = kThreads / 32;
-        finalize_bwd_kernel<<<(pb.C + per_block - 1) / per_block, kThreads, 0, stream>>>(
-            partials, pl.layout(), partials_v, pb.stat_plan.layout(), pb.C, pb.HW, invstd, dgamma, dbeta);
-    }
+                      (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, false>, pv.grid(), stream, in<T>(sp->xv),
+                              in<T>(sp->dyv), out<T>(nullptr), gamma, mean, invstd, pv.rows, pv.chunk, pv.tiles, pb.HW,
+                              pb.P, true, sink)));
+    launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
     // pass 2: the statistics terms, on S only
-    BwdParams bp{gamma, mean, invstd, dgamma, dbeta, static_cast<float>(1.0 / pb.s)};
+    const float inv_s = static_cast<float>(1.0 / pb.s);
     switch (pb.rule) {
     case BNS_RULE_FULL:
-        BNS_BY_TYPE_V(pb.dtype, pl.V, (launch_col_fixup<T, V>(pl, x, dy, dx, bp, nullptr, 0, pb.HW, pb.P, stream)));
+        BNS_BY_TYPE_V(pb.dtype, pl.V,
+                      (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pl.grid(), stream, in<T>(x), in<T>(dy),
+                              out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, static_cast<const int*>(nullptr), 0,
+                              pl.rows, pl.chunk, pl.tiles, pb.HW, pb.P)));
         break;
     case BNS_RULE_BATCH: {
         const int* list = nullptr;
         bns_status st = stage_list(pb, sp, ws, stream, &list);
         if (st != BNS_OK) return st;
-        const ColPlan& ps = pb.stat_plan;
-        BNS_BY_TYPE_V(pb.dtype, ps.V, (launch_col_fixup<T, V>(ps, x, dy, dx, bp, list, pb.begin, pb.HW, pb.P, stream)));
+        BNS_BY_TYPE_V(pb.dtype, pv.V,
+                      (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(x), in<T>(dy),
+                              out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, list, pb.begin, pv.rows, pv.chunk,
+                              pv.tiles, pb.HW, pb.P)));
         break;
     }
     case BNS_RULE_FEATURE: {
@@ -444,25 +437,17 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
         bns_status st = clear_status(pb, ws, stream, &status);
         if (st != BNS_OK) return st;
         const PatchPlan& pp = pb.patch_plan;
-        const unsigned grid = static_cast<unsigned>(pp.nchunks) * pb.C;
-        LaunchScope scope(BNS_KERNEL_PATCH_FIXUP, stream);
-        if (pb.dtype == BNS_F32)
-            patch_fixup_kernel<F32><<<grid, kThreads, 0, stream>>>(
-                static_cast<const float*>(x), static_cast<const float*>(dy), static_cast<float*>(dx), gamma, mean,
-                invstd, dgamma, dbeta, bp.inv_s, pb.patch, pb.N, pb.C, pb.H, pb.W, pp.chunk, status);
-        else
-            patch_fixup_kernel<BF16><<<grid, kThreads, 0, stream>>>(
-                static_cast<const unsigned short*>(x), static_cast<const unsigned short*>(dy),
-                static_cast<unsigned short*>(dx), gamma, mean, invstd, dgamma, dbeta, bp.inv_s, pb.patch, pb.N, pb.C,
-                pb.H, pb.W, pp.chunk, status);
+        BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, patch_fixup_kernel<T>, pp.grid(), stream, in<T>(x), in<T>(dy),
+                                      out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, pb.patch, pb.N, pb.C, pb.H,
+                                      pb.W, pp.chunk, pp.tiles, status)));
         break;
     }
     case BNS_RULE_VIRTUAL:
-        if (sp->dxv) {
-            const ColPlan& pv = pb.stat_plan;
+        if (sp->dxv)
             BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
-                          (launch_col_fixup<T, V>(pv, sp->xv, sp->dyv, sp->dxv, bp, nullptr, 0, pb.HW, pb.P, stream)));
-        }
+                          (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(sp->xv),
+                                  in<T>(sp->dyv), out<T>(sp->dxv), gamma, mean, invstd, dgamma, dbeta, inv_s,
+                                  static_cast<const int*>(nullptr), 0, pv.rows, pv.chunk, pv.tiles, pb.HW, pb.P)));
         break;
     }
     return last_error();
@@ -645,6 +630,28 @@ bns_status bns_profile_read(int kernel_kind, int* launches, float* total_ms) {
         *total_ms += ms;
     }
     return BNS_OK;
+}
+
+int bns_set_tuning(const char* name, int value) {
+    if (!name) return BNS_ERR_NULL;
+    struct Knob {
+        const char* name;
+        int* ivalue;
+        bool* bvalue;
+    } knobs[] = {{"target_blocks", &g_target_blocks, nullptr},   {"min_chunk", &g_min_chunk, nullptr},
+                 {"stat_target_blocks", &g_stat_target_blocks, nullptr}, {"stat_min_chunk", &g_stat_min_chunk, nullptr},
+                 {"pdl", nullptr, &g_pdl}};
+    for (const Knob& k : knobs) {
+        if (std::strcmp(name, k.name) != 0) continue;
+        if (k.ivalue) {
+            if (value < 1) return BNS_ERR_SHAPE;
+            *k.ivalue = value;
+        } else {
+            *k.bvalue = value != 0;
+        }
+        return BNS_OK;
+    }
+    return BNS_ERR_RULE;
 }
 
 const char* bns_kernel_name(int kernel_kind) {

@@ -7,7 +7,16 @@
 // is a full-width coalesced vector, and per-channel sums are kept per position in registers, so the
 // inner loop holds no index arithmetic, no shuffles and no shared memory.  Only after the loop are
 // the per-position sums folded into per-channel partials (one block-level pass through shared
-// memory), which a small "finalize" kernel combines across blocks in a fixed order.
+// memory), which a small "finalize" kernel (one warp per channel) combines in a fixed order.
+//
+// Feature Sampling uses the same scheme on a compacted position space: a sample row then has only
+// C*ph*pw positions (the patch elements of every map), thread j owns patch element j % (ph*pw) of
+// channel j / (ph*pw), and consecutive threads touch consecutive patch columns, rows and channels,
+// i.e. neighbouring addresses.
+//
+// Every kernel starts with a programmatic-dependent-launch wait, so that with the launch attribute
+// set its blocks may be scheduled while the previous kernel of the stream drains; nothing is read or
+// written before that wait.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -18,6 +27,12 @@ namespace bns {
 
 constexpr int kThreads = 256;  // threads per block of every streaming kernel
 constexpr int kUnroll = 4;     // rows in flight per thread
+
+// Programmatic dependent launch: wait until the preceding kernel of the stream has completed and
+// its writes are visible (a no-op when the launch did not ask for early scheduling).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Allow the next kernel of the stream to be scheduled once every block of this one got here.
+__device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
 
 // ------------------------------------------------------------------------------------ element types
 struct F32 {
@@ -160,16 +175,189 @@ struct TileChannels {
     }
 };
 
+// ------------------------------------------------------------------------------------ partials and how they are combined
+// How the partials of one pass are indexed: partial[(chunk*tiles + tile)*max_slots + slot], where
+// tile t covers positions [t*TP, (t+1)*TP) of a row and slot = channel - first channel of the tile.
+// The per-(chunk, channel) layout of the patch kernels is the case TP = HW, tiles = C, max_slots = 1.
+struct PartialLayout {
+    int nchunks;
+    unsigned tiles, TP;
+    int max_slots;
+    // partials that channel c receives: one per (row chunk, tile that meets the channel)
+    __device__ __forceinline__ int entries(int c, int HW, unsigned& t_lo, int& nt) const {
+        const unsigned pb = static_cast<unsigned>(c) * HW;
+        t_lo = pb / TP;
+        nt = static_cast<int>((pb + HW - 1) / TP - t_lo + 1);
+        return nchunks * nt;
+    }
+};
+
+// Statistics: where the partial moments are and where the finished mean / invstd go.
+struct StatsSink {
+    float4* partials;
+    PartialLayout L;
+    float inv_s, eps;
+    float* mean;
+    float* invstd;
+};
+
+// All partial moments of channel c, merged in a fixed order by one warp; mean / invstd written by lane 0.
+__device__ __forceinline__ void warp_finish_stats(const StatsSink& S, int c, int HW, int lane) {
+    unsigned t_lo;
+    int nt;
+    const int entries = S.L.entries(c, HW, t_lo, nt);
+    Moments acc = {0.f, 0.f, 0.f};
+    for (int e = lane; e < entries; e += 32) {
+        int ck = e / nt;
+        unsigned t = t_lo + static_cast<unsigned>(e - ck * nt);
+        int slot = c - static_cast<int>((t * S.L.TP) / static_cast<unsigned>(HW));
+        float4 v = S.partials[(static_cast<size_t>(ck) * S.L.tiles + t) * S.L.max_slots + slot];
+        acc = merge(acc, Moments{v.x, v.y, v.z});
+    }
+    acc = warp_merge(acc);
+    if (lane == 0) {
+        S.mean[c] = acc.mean;
+        S.invstd[c] = 1.0f / sqrtf(acc.m2 * S.inv_s + S.eps);
+    }
+}
+
+// Backward sums: partial (sum dy, sum dy (x - mean)) pairs of the real tensor and, when present, of the
+// virtual samples; both feed the same channel.
+struct GradSink {
+    float2* partials;
+    PartialLayout L;
+    float2* partials_v;  // NULL when no virtual gradient takes part
+    PartialLayout Lv;
+    const float* invstd;
+    float* dgamma;
+    float* dbeta;
+};
+
+__device__ __forceinline__ void warp_finish_grads(const GradSink& G, int c, int HW, int lane) {
+    float sum_dy = 0.f, sum_dyxc = 0.f;
+    for (int pass = 0; pass < 2; ++pass) {
+        const float2* src = pass ? G.partials_v : G.partials;
+        if (!src) continue;
+        const PartialLayout& Q = pass ? G.Lv : G.L;
+        unsigned t_lo;
+        int nt;
+        const int entries = Q.entries(c, HW, t_lo, nt);
+        for (int e = lane; e < entries; e += 32) {
+            int ck = e / nt;
+            unsigned t = t_lo + static_cast<unsigned>(e - ck * nt);
+            int slot = c - static_cast<int>((t * Q.TP) / static_cast<unsigned>(HW));
+            float2 v = src[(static_cast<size_t>(ck) * Q.tiles + t) * Q.max_slots + slot];
+            sum_dy += v.x;
+            sum_dyxc += v.y;
+        }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        sum_dy += __shfl_down_sync(0xffffffffu, sum_dy, d);
+        sum_dyxc += __shfl_down_sync(0xffffffffu, sum_dyxc, d);
+    }
+    if (lane == 0) {
+        G.dbeta[c] = sum_dy;
+        G.dgamma[c] = sum_dyxc * G.invstd[c];
+    }
+}
+
+// Folds the per-position moments of a block's tile (shared memory, one entry per position, every
+// position holding `cnt` values) into one partial per channel the tile meets.  The channel mean is the
+// plain average of the position means and M2 = sum(M2_q) + cnt * sum((mean_q - mean)^2): two passes of
+// plain sums, no divisions per element.  `span` is the number of positions per channel.
+__device__ __forceinline__ void fold_moments(const float* s_mean, const float* s_m2, float cnt, const TileChannels& tc,
+                                             int span, float4* out) {
+    if (span >= 32) {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int slot = warp; slot < tc.nslots; slot += kThreads / 32) {
+            unsigned lo, hi;
+            tc.range(slot, span, lo, hi);
+            float sum = 0.f;
+            for (unsigned q = lo + lane; q < hi; q += 32) sum += s_mean[q];
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+            const float len = static_cast<float>(hi - lo);
+            const float mu = sum / len;
+            float dev = 0.f, m2 = 0.f;
+            for (unsigned q = lo + lane; q < hi; q += 32) {
+                float d = s_mean[q] - mu;
+                dev = fmaf(d, d, dev);
+                m2 += s_m2[q];
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                dev += __shfl_xor_sync(0xffffffffu, dev, d);
+                m2 += __shfl_xor_sync(0xffffffffu, m2, d);
+            }
+            if (lane == 0) out[slot] = make_float4(cnt * len, mu, fmaf(cnt, dev, m2), 0.f);
+        }
+    } else {
+        // fewer positions per channel than a warp has lanes: one thread per channel
+        for (int slot = threadIdx.x; slot < tc.nslots; slot += kThreads) {
+            unsigned lo, hi;
+            tc.range(slot, span, lo, hi);
+            float sum = 0.f;
+            for (unsigned q = lo; q < hi; ++q) sum += s_mean[q];
+            const float len = static_cast<float>(hi - lo);
+            const float mu = sum / len;
+            float dev = 0.f, m2 = 0.f;
+            for (unsigned q = lo; q < hi; ++q) {
+                float d = s_mean[q] - mu;
+                dev = fmaf(d, d, dev);
+                m2 += s_m2[q];
+            }
+            out[slot] = make_float4(cnt * len, mu, fmaf(cnt, dev, m2), 0.f);
+        }
+    }
+}
+
+// The same for plain sums (backward): one (sum dy, sum dy (x - mean)) pair per channel the tile meets.
+__device__ __forceinline__ void fold_sums(const float* s_a, const float* s_b, const TileChannels& tc, int span,
+                                          float2* out) {
+    if (span >= 32) {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int slot = warp; slot < tc.nslots; slot += kThreads / 32) {
+            unsigned lo, hi;
+            tc.range(slot, span, lo, hi);
+            float sa = 0.f, sb = 0.f;
+            for (unsigned q = lo + lane; q < hi; q += 32) {
+                sa += s_a[q];
+                sb += s_b[q];
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                sa += __shfl_down_sync(0xffffffffu, sa, d);
+                sb += __shfl_down_sync(0xffffffffu, sb, d);
+            }
+            if (lane == 0) out[slot] = make_float2(sa, sb);
+        }
+    } else {
+        for (int slot = threadIdx.x; slot < tc.nslots; slot += kThreads) {
+            unsigned lo, hi;
+            tc.range(slot, span, lo, hi);
+            float sa = 0.f, sb = 0.f;
+            for (unsigned q = lo; q < hi; ++q) {
+                sa += s_a[q];
+                sb += s_b[q];
+            }
+            out[slot] = make_float2(sa, sb);
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------ statistics over whole samples
 // Partial moments of x[list, :] per (row chunk, tile, channel slot).  `list` (device) holds the
 // sample indices or is NULL for the contiguous range begin .. begin+count-1.
 template <typename T, int V>
 __global__ void __launch_bounds__(kThreads)
 col_moments_kernel(const typename T::storage* __restrict__ x, const int* __restrict__ list, int begin, int count,
-                   int chunk, unsigned tiles, int HW, unsigned P, int max_slots, float4* __restrict__ partials) {
+                   int chunk, unsigned tiles, int HW, unsigned P, StatsSink S) {
     constexpr unsigned TP = kThreads * V;
     __shared__ float s_mean[TP];
     __shared__ float s_m2[TP];
+    grid_dependency_wait();
+    grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
     const unsigned ck = blockIdx.x / tiles;
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
@@ -180,7 +368,7 @@ col_moments_kernel(const typename T::storage* __restrict__ x, const int* __restr
     for (int j = 0; j < V; ++j) K[j] = s1[j] = s2[j] = 0.f;
     if (p < P) {
         const typename T::storage* xp = x + p;
-        {
+        {   // pivot: the first value of every position (its own deviation is zero)
             int n = list ? list[i0] : begin + i0;
             Vec<T, V> v;
             v.load(xp + static_cast<size_t>(n) * P);
@@ -223,27 +411,8 @@ col_moments_kernel(const typename T::storage* __restrict__ x, const int* __restr
         s_m2[threadIdx.x * V + j] = m.m2;
     }
     __syncthreads();
-    const TileChannels tc(tile, TP, P, HW);
-    float4* out = partials + (static_cast<size_t>(ck) * tiles + tile) * max_slots;
-    if (HW >= 32) {
-        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-        for (int slot = warp; slot < tc.nslots; slot += kThreads / 32) {
-            unsigned lo, hi;
-            tc.range(slot, HW, lo, hi);
-            Moments acc = {0.f, 0.f, 0.f};
-            for (unsigned q = lo + lane; q < hi; q += 32) acc = merge(acc, Moments{cnt, s_mean[q], s_m2[q]});
-            acc = warp_merge(acc);
-            if (lane == 0) out[slot] = make_float4(acc.cnt, acc.mean, acc.m2, 0.f);
-        }
-    } else {
-        for (int slot = threadIdx.x; slot < tc.nslots; slot += kThreads) {
-            unsigned lo, hi;
-            tc.range(slot, HW, lo, hi);
-            Moments acc = {0.f, 0.f, 0.f};
-            for (unsigned q = lo; q < hi; ++q) acc = merge(acc, Moments{cnt, s_mean[q], s_m2[q]});
-            out[slot] = make_float4(acc.cnt, acc.mean, acc.m2, 0.f);
-        }
-    }
+    fold_moments(s_mean, s_m2, cnt, TileChannels(tile, TP, P, HW), HW,
+                 S.partials + (static_cast<size_t>(ck) * tiles + tile) * S.L.max_slots);
 }
 
 // ------------------------------------------------------------------------------------ statistics over patches
@@ -270,123 +439,103 @@ __device__ __forceinline__ void patch_origin(const PatchRule& r, int n, int c, i
     if ((oh != o.x || ow != o.y) && status) atomicOr(status, 1u);
 }
 
-// One block per (sample chunk, channel): threads stride over the patch elements of the chunk's maps.
+// A thread of the patch kernels owns compact position j of every sample row: patch element
+// e = j % (ph*pw) (row e / pw, column e % pw of the patch) of channel c = j / (ph*pw).
+struct PatchThread {
+    int c, row, col;
+    size_t plane;  // c*H*W + row*W + col: offset inside a sample row, before the patch origin is added
+    __device__ __forceinline__ PatchThread(unsigned j, const PatchRule& r, int H, int W) {
+        const int PP = r.ph * r.pw;
+        c = static_cast<int>(j / static_cast<unsigned>(PP));
+        const int e = static_cast<int>(j - static_cast<unsigned>(c) * PP);
+        row = e / r.pw;
+        col = e - row * r.pw;
+        plane = static_cast<size_t>(c) * H * W + static_cast<size_t>(row) * W + col;
+    }
+    // element offset of this thread's patch element in sample n
+    __device__ __forceinline__ size_t at(const PatchRule& r, int n, size_t P, int H, int W, unsigned* status) const {
+        int oh, ow;
+        patch_origin(r, n, c, H, W, status, oh, ow);
+        return static_cast<size_t>(n) * P + plane + static_cast<size_t>(oh) * W + ow;
+    }
+};
+
+// Partial moments of the patch elements per (sample chunk, tile of compact positions, channel slot).
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 patch_moments_kernel(const typename T::storage* __restrict__ x, PatchRule rule, int N, int C, int H, int W, int chunk,
-                     float4* __restrict__ partials, unsigned* status) {
-    __shared__ Moments s_warp[kThreads / 32];
-    const int c = blockIdx.x % C;
-    const int ck = blockIdx.x / C;
-    const int n0 = ck * chunk, n1 = min(N, n0 + chunk);
+                     unsigned tiles, StatsSink S, unsigned* status) {
+    __shared__ float s_mean[kThreads];
+    __shared__ float s_m2[kThreads];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const unsigned tile = blockIdx.x % tiles;
+    const unsigned ck = blockIdx.x / tiles;
     const int PP = rule.ph * rule.pw;
-    const int total = (n1 - n0) * PP;
-    const size_t HW = static_cast<size_t>(H) * W;
-    float K = 0.f, s1 = 0.f, s2 = 0.f, cnt = 0.f;
-    for (int q = threadIdx.x; q < total; q += kThreads) {
-        int nl = q / PP, e = q - nl * PP;
-        int r = e / rule.pw, col = e - r * rule.pw;
-        int n = n0 + nl, oh, ow;
-        patch_origin(rule, n, c, H, W, status, oh, ow);
-        float v = to_float<T>(x[(static_cast<size_t>(n) * C + c) * HW + static_cast<size_t>(oh + r) * W + ow + col]);
-        if (cnt == 0.f) K = v;
-        float d = v - K;
-        s1 += d;
-        s2 = fmaf(d, d, s2);
-        cnt += 1.f;
-    }
-    Moments m = warp_merge(from_shifted_sums(cnt, K, s1, s2));
-    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = m;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        Moments acc = s_warp[0];
-        for (int w = 1; w < kThreads / 32; ++w) acc = merge(acc, s_warp[w]);
-        partials[static_cast<size_t>(ck) * C + c] = make_float4(acc.cnt, acc.mean, acc.m2, 0.f);
-    }
-}
-
-// ------------------------------------------------------------------------------------ finalize
-// How the partials of one pass are indexed: partial[(chunk*tiles + tile)*max_slots + slot], where
-// tile t covers positions [t*TP, (t+1)*TP) of a row and slot = channel - first channel of the tile.
-// The per-(chunk, channel) layout of the patch kernels is the case TP = HW, tiles = C, max_slots = 1.
-struct PartialLayout {
-    int nchunks;
-    unsigned tiles, TP;
-    int max_slots;
-};
-
-// One warp per channel merges its partial moments in a fixed order and writes mean and invstd.
-__global__ void __launch_bounds__(kThreads)
-finalize_stats_kernel(const float4* __restrict__ partials, PartialLayout L, int C, int HW, float s, float eps,
-                      float* __restrict__ mean, float* __restrict__ invstd) {
-    const int c = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (c >= C) return;
-    const unsigned pb = static_cast<unsigned>(c) * HW;
-    const unsigned t_lo = pb / L.TP, t_hi = (pb + HW - 1) / L.TP;
-    const int nt = static_cast<int>(t_hi - t_lo + 1);
-    const int entries = L.nchunks * nt;
-    Moments acc = {0.f, 0.f, 0.f};
-    for (int e = lane; e < entries; e += 32) {
-        int ck = e / nt;
-        unsigned t = t_lo + static_cast<unsigned>(e - ck * nt);
-        int slot = c - static_cast<int>((t * L.TP) / static_cast<unsigned>(HW));
-        float4 v = partials[(static_cast<size_t>(ck) * L.tiles + t) * L.max_slots + slot];
-        acc = merge(acc, Moments{v.x, v.y, v.z});
-    }
-    acc = warp_merge(acc);
-    if (lane == 0) {
-        float var = acc.m2 / s;
-        mean[c] = acc.mean;
-        invstd[c] = 1.0f / sqrtf(var + eps);
-    }
-}
-
-// One warp per channel adds its partial (sum dy, sum dy (x - mean)) pairs in a fixed order, from the
-// real tensor and, when present, from the virtual samples.
-__global__ void __launch_bounds__(kThreads)
-finalize_bwd_kernel(const float2* __restrict__ partials, PartialLayout L, const float2* __restrict__ partials_v,
-                    PartialLayout Lv, int C, int HW, const float* __restrict__ invstd, float* __restrict__ dgamma,
-                    float* __restrict__ dbeta) {
-    const int c = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (c >= C) return;
-    const unsigned pb = static_cast<unsigned>(c) * HW;
-    float sum_dy = 0.f, sum_dyxc = 0.f;
-    for (int pass = 0; pass < 2; ++pass) {
-        const float2* src = pass ? partials_v : partials;
-        if (!src) continue;
-        const PartialLayout& Q = pass ? Lv : L;
-        const unsigned t_lo = pb / Q.TP, t_hi = (pb + HW - 1) / Q.TP;
-        const int nt = static_cast<int>(t_hi - t_lo + 1);
-        const int entries = Q.nchunks * nt;
-        for (int e = lane; e < entries; e += 32) {
-            int ck = e / nt;
-            unsigned t = t_lo + static_cast<unsigned>(e - ck * nt);
-            int slot = c - static_cast<int>((t * Q.TP) / static_cast<unsigned>(HW));
-            float2 v = src[(static_cast<size_t>(ck) * Q.tiles + t) * Q.max_slots + slot];
-            sum_dy += v.x;
-            sum_dyxc += v.y;
+    const unsigned Pc = static_cast<unsigned>(C) * PP;  // compact positions per sample
+    const unsigned j = tile * kThreads + threadIdx.x;
+    const size_t P = static_cast<size_t>(C) * H * W;
+    const int n0 = ck * chunk, n1 = min(N, n0 + chunk);
+    const float cnt = static_cast<float>(n1 - n0);
+    float K = 0.f, s1 = 0.f, s2 = 0.f;
+    if (j < Pc) {
+        const PatchThread me(j, rule, H, W);
+        K = to_float<T>(x[me.at(rule, n0, P, H, W, status)]);  // pivot: the first value
+        int n = n0 + 1;
+        for (; n + kUnroll <= n1; n += kUnroll) {
+            float v[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) v[u] = to_float<T>(x[me.at(rule, n + u, P, H, W, status)]);
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                float d = v[u] - K;
+                s1 += d;
+                s2 = fmaf(d, d, s2);
+            }
+        }
+        for (; n < n1; ++n) {
+            float d = to_float<T>(x[me.at(rule, n, P, H, W, status)]) - K;
+            s1 += d;
+            s2 = fmaf(d, d, s2);
         }
     }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-        sum_dy += __shfl_down_sync(0xffffffffu, sum_dy, d);
-        sum_dyxc += __shfl_down_sync(0xffffffffu, sum_dyxc, d);
-    }
-    if (lane == 0) {
-        dbeta[c] = sum_dy;
-        dgamma[c] = sum_dyxc * invstd[c];
-    }
+    Moments m = from_shifted_sums(cnt, K, s1, s2);
+    s_mean[threadIdx.x] = m.mean;
+    s_m2[threadIdx.x] = m.m2;
+    __syncthreads();
+    fold_moments(s_mean, s_m2, cnt, TileChannels(tile, kThreads, Pc, PP), PP,
+                 S.partials + (static_cast<size_t>(ck) * tiles + tile) * S.L.max_slots);
+}
+
+// ------------------------------------------------------------------------------------ finalize kernels
+// One warp per channel; used when the producers did not combine the partials themselves.
+__global__ void __launch_bounds__(kThreads)
+finalize_stats_kernel(StatsSink S, int C, int HW) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (c >= C) return;
+    warp_finish_stats(S, c, HW, threadIdx.x & 31);
+}
+
+__global__ void __launch_bounds__(kThreads)
+finalize_bwd_kernel(GradSink G, int C, int HW) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (c >= C) return;
+    warp_finish_grads(G, c, HW, threadIdx.x & 31);
 }
 
 // ------------------------------------------------------------------------------------ normalise + affine
-// y = a_c x + b_c with a_c = gamma_c invstd_c and b_c = beta_c - mean_c a_c, over rows [n0, n1).
+// y = a_c x + b_c with a_c = gamma_c invstd_c and b_c = beta_c - mean_c a_c, over the rows of the chunk.
 template <typename T, int V>
 __global__ void __launch_bounds__(kThreads)
 col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::storage* __restrict__ y,
                      const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
                      const float* __restrict__ invstd, int rows, int chunk, unsigned tiles, int HW, unsigned P) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
     const unsigned ck = blockIdx.x / tiles;
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
@@ -437,10 +586,12 @@ __global__ void __launch_bounds__(kThreads)
 col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
                       typename T::storage* __restrict__ dx, const float* __restrict__ gamma,
                       const float* __restrict__ mean, const float* __restrict__ invstd, int rows, int chunk,
-                      unsigned tiles, int HW, unsigned P, int max_slots, float2* __restrict__ partials) {
+                      unsigned tiles, int HW, unsigned P, bool virtual_pass, GradSink G) {
     constexpr unsigned TP = kThreads * V;
     __shared__ float s_dy[TP];
     __shared__ float s_dyxc[TP];
+    grid_dependency_wait();
+    grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
     const unsigned ck = blockIdx.x / tiles;
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
@@ -511,37 +662,9 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
         s_dyxc[threadIdx.x * V + j] = acc_dyxc[j];
     }
     __syncthreads();
-    const TileChannels tc(tile, TP, P, HW);
-    float2* out = partials + (static_cast<size_t>(ck) * tiles + tile) * max_slots;
-    if (HW >= 32) {
-        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-        for (int slot = warp; slot < tc.nslots; slot += kThreads / 32) {
-            unsigned lo, hi;
-            tc.range(slot, HW, lo, hi);
-            float sa = 0.f, sb = 0.f;
-            for (unsigned q = lo + lane; q < hi; q += 32) {
-                sa += s_dy[q];
-                sb += s_dyxc[q];
-            }
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                sa += __shfl_down_sync(0xffffffffu, sa, d);
-                sb += __shfl_down_sync(0xffffffffu, sb, d);
-            }
-            if (lane == 0) out[slot] = make_float2(sa, sb);
-        }
-    } else {
-        for (int slot = threadIdx.x; slot < tc.nslots; slot += kThreads) {
-            unsigned lo, hi;
-            tc.range(slot, HW, lo, hi);
-            float sa = 0.f, sb = 0.f;
-            for (unsigned q = lo; q < hi; ++q) {
-                sa += s_dy[q];
-                sb += s_dyxc[q];
-            }
-            out[slot] = make_float2(sa, sb);
-        }
-    }
+    float2* out = (virtual_pass ? G.partials_v : G.partials) +
+                  (static_cast<size_t>(ck) * tiles + tile) * (virtual_pass ? G.Lv.max_slots : G.L.max_slots);
+    fold_sums(s_dy, s_dyxc, TileChannels(tile, TP, P, HW), HW, out);
 }
 
 // ------------------------------------------------------------------------------------ backward, statistics terms
@@ -551,14 +674,13 @@ struct FixCoef {
     float a, A, Q, mu;
 };
 
-__device__ __forceinline__ FixCoef fix_coef(int c, const float* gamma, const float* mean, const float* invstd,
-                                            const float* dgamma, const float* dbeta, float inv_s) {
+__device__ __forceinline__ FixCoef fix_coef(float gamma, float mean, float invstd, float dgamma, float dbeta,
+                                            float inv_s) {
     FixCoef k;
-    float is = invstd[c];
-    k.a = gamma[c] * is;
-    k.A = k.a * dbeta[c] * inv_s;
-    k.Q = k.a * is * dgamma[c] * inv_s;
-    k.mu = mean[c];
+    k.a = gamma * invstd;
+    k.A = k.a * dbeta * inv_s;
+    k.Q = k.a * invstd * dgamma * inv_s;
+    k.mu = mean;
     return k;
 }
 
@@ -570,6 +692,8 @@ col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::st
                  const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
                  float inv_s, const int* __restrict__ list, int begin, int count, int chunk, unsigned tiles, int HW,
                  unsigned P) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
     const unsigned ck = blockIdx.x / tiles;
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
@@ -579,22 +703,22 @@ col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::st
         int c[V];
         position_channels<V>(p, HW, c);
 #pragma unroll
-        for (int j = 0; j < V; ++j) k[j] = fix_coef(c[j], gamma, mean, invstd, dgamma, dbeta, inv_s);
+        for (int j = 0; j < V; ++j) k[j] = fix_coef(gamma[c[j]], mean[c[j]], invstd[c[j]], dgamma[c[j]], dbeta[c[j]], inv_s);
     }
     const int i0 = ck * chunk, i1 = min(count, i0 + chunk);
     int i = i0;
-    for (; i + 2 <= i1; i += 2) {
-        Vec<T, V> vx[2], vg[2];
-        size_t off[2];
+    for (; i + kUnroll <= i1; i += kUnroll) {
+        Vec<T, V> vx[kUnroll], vg[kUnroll];
+        size_t off[kUnroll];
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
+        for (int u = 0; u < kUnroll; ++u) {
             int n = list ? list[i + u] : begin + i + u;
             off[u] = static_cast<size_t>(n) * P + p;
             vx[u].load(x + off[u]);
             if (dy) vg[u].load(dy + off[u]);
         }
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
+        for (int u = 0; u < kUnroll; ++u) {
 #pragma unroll
             for (int j = 0; j < V; ++j) {
                 float g = dy ? vg[u].get(j) : 0.f;
@@ -618,28 +742,40 @@ col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::st
     }
 }
 
-// The same for the patch elements of the chunk's maps of one channel.
+// The same for the patch elements (compact positions, see PatchThread).
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
                    typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
                    const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
-                   float inv_s, PatchRule rule, int N, int C, int H, int W, int chunk, unsigned* status) {
-    const int c = blockIdx.x % C;
-    const int ck = blockIdx.x / C;
+                   float inv_s, PatchRule rule, int N, int C, int H, int W, int chunk, unsigned tiles,
+                   unsigned* status) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const unsigned tile = blockIdx.x % tiles;
+    const unsigned ck = blockIdx.x / tiles;
+    const unsigned j = tile * kThreads + threadIdx.x;
+    if (j >= static_cast<unsigned>(C) * rule.ph * rule.pw) return;
+    const PatchThread me(j, rule, H, W);
+    const size_t P = static_cast<size_t>(C) * H * W;
+    const FixCoef k = fix_coef(gamma[me.c], mean[me.c], invstd[me.c], dgamma[me.c], dbeta[me.c], inv_s);
     const int n0 = ck * chunk, n1 = min(N, n0 + chunk);
-    const int PP = rule.ph * rule.pw;
-    const int total = (n1 - n0) * PP;
-    const size_t HW = static_cast<size_t>(H) * W;
-    const FixCoef k = fix_coef(c, gamma, mean, invstd, dgamma, dbeta, inv_s);
-    for (int q = threadIdx.x; q < total; q += kThreads) {
-        int nl = q / PP, e = q - nl * PP;
-        int r = e / rule.pw, col = e - r * rule.pw;
-        int n = n0 + nl, oh, ow;
-        patch_origin(rule, n, c, H, W, status, oh, ow);
-        size_t at = (static_cast<size_t>(n) * C + c) * HW + static_cast<size_t>(oh + r) * W + ow + col;
-        float g = to_float<T>(dy[at]);
-        float xv = to_float<T>(x[at]);
+    int n = n0;
+    for (; n + kUnroll <= n1; n += kUnroll) {
+        size_t at[kUnroll];
+        float g[kUnroll], xv[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            at[u] = me.at(rule, n + u, P, H, W, status);
+            g[u] = to_float<T>(dy[at[u]]);
+            xv[u] = to_float<T>(x[at[u]]);
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) dx[at[u]] = from_float<T>(fmaf(k.a, g[u], -k.A) - k.Q * (xv[u] - k.mu));
+    }
+    for (; n < n1; ++n) {
+        size_t at = me.at(rule, n, P, H, W, status);
+        float g = to_float<T>(dy[at]), xv = to_float<T>(x[at]);
         dx[at] = from_float<T>(fmaf(k.a, g, -k.A) - k.Q * (xv - k.mu));
     }
 }
@@ -648,6 +784,7 @@ patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::
 __global__ void __launch_bounds__(kThreads)
 selection_mask_kernel(uint8_t* __restrict__ mask, int rule, const int* __restrict__ list, int begin, int count,
                       PatchRule patch, int N, int C, int H, int W, unsigned* status) {
+    grid_dependency_wait();
     const size_t total = static_cast<size_t>(N) * C * H * W;
     for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < total;
          i += static_cast<size_t>(gridDim.x) * kThreads) {

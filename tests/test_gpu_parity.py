@@ -180,3 +180,39 @@ def test_bad_device_offsets_raise_flag_and_stay_in_bounds():
     case.offsets = clamped
     f = O.forward(case.x, case.gamma, case.beta, 1e-5, case.oracle_sampling())
     np.testing.assert_allclose(mean.cpu().numpy(), f.mean, atol=1e-5)
+
+
+# ----------------------------------------------------------------------------- launch-shape knobs change no bits they should not
+@pytest.mark.parametrize("rule,kw", [
+    ("batch", dict(k=6)), ("feature", dict(ph=3, pw=3, offset_mode=2)), ("virtual", dict(nv=2)), ("full", dict()),
+])
+def test_programmatic_dependent_launch_changes_nothing(rule, kw):
+    """With and without programmatic dependent launch the kernels run the same arithmetic in the same
+    order, so the results must be identical bit for bit."""
+    import torch
+    from paper_1810_10962_b200 import bns
+    case = make_case(40, 24, 20, 20, rule, seed=85, **kw)
+    try:
+        bns.set_tuning("pdl", 0)
+        a = run_gpu(case)
+    finally:
+        bns.set_tuning("pdl", 1)
+    b = run_gpu(case)
+    compare(case, b)
+    for key in a.raw:
+        assert torch.equal(a.raw[key], b.raw[key]), key
+
+
+@pytest.mark.parametrize("target", [37, 148, 4736])
+def test_other_grid_shapes_still_match_the_oracle(target):
+    """Splitting the rows into more or fewer chunks reorders sums but must stay within tolerance."""
+    from paper_1810_10962_b200 import bns
+    try:
+        bns.set_tuning("target_blocks", target)
+        bns.set_tuning("stat_target_blocks", target)
+        for rule, kw in [("batch", dict(k=9)), ("feature", dict(ph=5, pw=3)), ("full", dict())]:
+            case = make_case(70, 12, 33, 31, rule, seed=86, **kw)
+            compare(case, run_gpu(case))
+    finally:
+        bns.set_tuning("target_blocks", 148 * 8)
+        bns.set_tuning("stat_target_blocks", 148 * 8)
