@@ -37,9 +37,10 @@ import bns_inputs as I  # noqa: E402
 EPS = 1e-5
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one col_bwd_reduce_kernel launch on the default workload,
-# from the ncu capture summarised in profiles/; None while no capture of the current kernel exists.
-BWD_REDUCE_DRAM_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one col_bwd_reduce_kernel<F32,4,true> launch on the default
+# workload's layer shape (256x64x56x56 fp32), from the ncu capture summarised in
+# profiles/col_bwd_reduce_f32_resnet18_stage1.md; reported only for that workload.
+BWD_REDUCE_DRAM_TRAFFIC_BYTES = 579_660_800   # 411.13 MB read + 168.53 MB written (rest of dx still dirty in L2)
 
 
 # ----------------------------------------------------------------------------- workloads
@@ -354,7 +355,8 @@ def run_ours(args):
         algo = sum(l.count * 3 * l.elems * l.ebytes for l in layers) / launches_per_step
         achieved = algo / (kt["avg_us"] * 1e-6) / 1e9
         roofline = {"kernel": "col_bwd_reduce_kernel", "bound": "hbm", "achieved": round(achieved, 1), "peak": peak,
-                    "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": BWD_REDUCE_DRAM_TRAFFIC_BYTES,
+                    "unit": "GB/s", "frac": round(achieved / peak, 4),
+                    "traffic": BWD_REDUCE_DRAM_TRAFFIC_BYTES if args.workload == "resnet18_stage1" else None,
                     "algorithmic_bytes_per_launch": int(algo), "avg_launch_us": kt["avg_us"], "peak_source": peak_source,
                     "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4)}
 

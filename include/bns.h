@@ -184,7 +184,8 @@ const char* bns_kernel_name(int kernel_kind);
 /* Launch-shape knobs (process-wide; change them only while no call is in flight, and recompute
  * bns_workspace_bytes afterwards).  "target_blocks" / "min_chunk": blocks per launch and least rows
  * per block of the streaming kernels; "stat_target_blocks" / "stat_min_chunk": the same for the
- * statistics kernels; "pdl": 0/1 programmatic dependent launch.  Returns BNS_OK,
+ * statistics kernels; "pdl": 0/1 programmatic dependent launch; "l2_order": 0/1 visit rows in an
+ * order that lets a kernel find in L2 what the previous one read.  Returns BNS_OK,
  * BNS_ERR_RULE for an unknown name or BNS_ERR_SHAPE for a value < 1. */
 int bns_set_tuning(const char* name, int value);
 

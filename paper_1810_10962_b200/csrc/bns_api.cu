@@ -79,8 +79,8 @@ struct ColPlan {
     size_t partial_count() const { return static_cast<size_t>(nchunks) * tiles * max_slots; }
 };
 
-int g_target_blocks = kSmCount * 8;       // streaming kernels: blocks per launch aimed at when splitting the rows
-int g_min_chunk = 4;                      // ... but at least this many rows per block
+int g_target_blocks = kSmCount * 32;      // streaming kernels: blocks per launch aimed at when splitting the rows
+int g_min_chunk = 8;                      // ... but at least this many rows per block
 int g_stat_target_blocks = kSmCount * 8;  // short statistics kernels: one wave of blocks, all loads in flight
 int g_stat_min_chunk = 1;
 
@@ -279,6 +279,7 @@ bns_status clear_status(const Problem& pb, void* ws, cudaStream_t stream, unsign
 
 // ------------------------------------------------------------------------------------ launches
 bool g_pdl = true;    // ask for programmatic dependent launch (blocks may be scheduled while the previous kernel drains)
+bool g_l2_order = true;  // order rows so that a kernel re-reads what the previous one left in L2
 
 template <typename... KArgs, typename... Args>
 void launch(int kind, void (*kernel)(KArgs...), unsigned grid, cudaStream_t s, Args&&... args) {
@@ -351,7 +352,7 @@ bns_status run_statistics(const Problem& pb, const bns_sampling* sp, const void*
         sink.L = pp.layout();
         span = pb.patch.ph * pb.patch.pw;
         BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_MOMENTS, patch_moments_kernel<T>, pp.grid(), stream, in<T>(x),
-                                      pb.patch, pb.N, pb.C, pb.H, pb.W, pp.chunk, pp.tiles, sink, status)));
+                                      pb.patch, pb.N, pb.C, pb.H, pb.W, pp.nchunks, pp.tiles, sink, status)));
     } else {
         const int* list = nullptr;
         bns_status st = stage_list(pb, sp, ws, stream, &list);
@@ -363,7 +364,7 @@ bns_status run_statistics(const Problem& pb, const bns_sampling* sp, const void*
         sink.L = pl.layout();
         BNS_BY_TYPE_V(dt, pl.V,
                       (launch(BNS_KERNEL_COL_MOMENTS, col_moments_kernel<T, V>, pl.grid(), stream, in<T>(data), list, begin,
-                              pl.rows, pl.chunk, pl.tiles, pb.HW, pb.P, sink)));
+                              pl.rows, pl.nchunks, pl.tiles, pb.HW, pb.P, sink)));
     }
     launch(BNS_KERNEL_FINALIZE_STATS, finalize_stats_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, span);
     return last_error();
@@ -374,14 +375,20 @@ bns_status forward_impl(const Problem& pb, const bns_sampling* sp, const void* x
     bns_status st = run_statistics(pb, sp, x, eps, mean, invstd, ws, stream);
     if (st != BNS_OK) return st;
     const ColPlan& pl = pb.main_plan;
+    // visit first the rows that the statistics kernel has just read: they are still in L2
+    RowOrder order{RowOrder::kIdentity, pb.N, 0, 0};
+    if (g_l2_order && pb.rule == BNS_RULE_FULL) order.mode = RowOrder::kReversed;
+    if (g_l2_order && pb.rule == BNS_RULE_BATCH && pb.contiguous)
+        order = RowOrder{RowOrder::kRangeFirst, pb.N, pb.begin, pb.count};
     BNS_BY_TYPE_V(pb.dtype, pl.V,
                   (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pl.grid(), stream, in<T>(x), out<T>(y), gamma,
-                          beta, mean, invstd, pl.rows, pl.chunk, pl.tiles, pb.HW, pb.P)));
+                          beta, mean, invstd, order, pl.nchunks, pl.tiles, pb.HW, pb.P)));
     if (pb.rule == BNS_RULE_VIRTUAL && sp->yv) {
         const ColPlan& pv = pb.stat_plan;
         BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
                       (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pv.grid(), stream, in<T>(sp->xv),
-                              out<T>(sp->yv), gamma, beta, mean, invstd, pv.rows, pv.chunk, pv.tiles, pb.HW, pb.P)));
+                              out<T>(sp->yv), gamma, beta, mean, invstd, RowOrder{RowOrder::kIdentity, pv.rows, 0, 0},
+                              pv.nchunks, pv.tiles, pb.HW, pb.P)));
     }
     return last_error();
 }
@@ -396,22 +403,27 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
     GradSink sink{ws_at<float2>(ws, pb.off_bwd), pl.layout(), virtual_grads ? ws_at<float2>(ws, pb.off_bwd_v) : nullptr,
                   pv.layout(), invstd, dgamma, dbeta};
     // pass 1: the sums of Eq. 5 over every real element; dx = gamma invstd dy everywhere unless every
-    // element is sampled (FULL), where the second pass writes dx anyway.
+    // element is sampled (FULL), where the second pass writes dx anyway.  The rows that the second pass
+    // reads again are visited last, so that it finds them in L2.
+    RowOrder order{RowOrder::kIdentity, pb.N, 0, 0};
+    if (g_l2_order && pb.rule == BNS_RULE_BATCH && pb.contiguous)
+        order = RowOrder{RowOrder::kRangeLast, pb.N, pb.begin, pb.count};
     if (full)
         BNS_BY_TYPE_V(pb.dtype, pl.V,
                       (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, false>, pl.grid(), stream, in<T>(x),
-                              in<T>(dy), out<T>(nullptr), gamma, mean, invstd, pl.rows, pl.chunk, pl.tiles, pb.HW, pb.P,
+                              in<T>(dy), out<T>(nullptr), gamma, mean, invstd, order, pl.nchunks, pl.tiles, pb.HW, pb.P,
                               false, sink)));
     else
         BNS_BY_TYPE_V(pb.dtype, pl.V,
                       (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, true>, pl.grid(), stream, in<T>(x),
-                              in<T>(dy), out<T>(dx), gamma, mean, invstd, pl.rows, pl.chunk, pl.tiles, pb.HW, pb.P, false,
+                              in<T>(dy), out<T>(dx), gamma, mean, invstd, order, pl.nchunks, pl.tiles, pb.HW, pb.P, false,
                               sink)));
     if (virtual_grads)
         BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
                       (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, false>, pv.grid(), stream, in<T>(sp->xv),
-                              in<T>(sp->dyv), out<T>(nullptr), gamma, mean, invstd, pv.rows, pv.chunk, pv.tiles, pb.HW,
-                              pb.P, true, sink)));
+                              in<T>(sp->dyv), out<T>(nullptr), gamma, mean, invstd,
+                              RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P, true,
+                              sink)));
     launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
     // pass 2: the statistics terms, on S only
     const float inv_s = static_cast<float>(1.0 / pb.s);
@@ -420,7 +432,8 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
         BNS_BY_TYPE_V(pb.dtype, pl.V,
                       (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pl.grid(), stream, in<T>(x), in<T>(dy),
                               out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, static_cast<const int*>(nullptr), 0,
-                              pl.rows, pl.chunk, pl.tiles, pb.HW, pb.P)));
+                              RowOrder{g_l2_order ? RowOrder::kReversed : RowOrder::kIdentity, pl.rows, 0, 0}, pl.nchunks,
+                              pl.tiles, pb.HW, pb.P)));
         break;
     case BNS_RULE_BATCH: {
         const int* list = nullptr;
@@ -428,8 +441,8 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
         if (st != BNS_OK) return st;
         BNS_BY_TYPE_V(pb.dtype, pv.V,
                       (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(x), in<T>(dy),
-                              out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, list, pb.begin, pv.rows, pv.chunk,
-                              pv.tiles, pb.HW, pb.P)));
+                              out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, list, pb.begin,
+                              RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P)));
         break;
     }
     case BNS_RULE_FEATURE: {
@@ -439,7 +452,7 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
         const PatchPlan& pp = pb.patch_plan;
         BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, patch_fixup_kernel<T>, pp.grid(), stream, in<T>(x), in<T>(dy),
                                       out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, pb.patch, pb.N, pb.C, pb.H,
-                                      pb.W, pp.chunk, pp.tiles, status)));
+                                      pb.W, pp.nchunks, pp.tiles, status)));
         break;
     }
     case BNS_RULE_VIRTUAL:
@@ -447,7 +460,8 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
             BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
                           (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(sp->xv),
                                   in<T>(sp->dyv), out<T>(sp->dxv), gamma, mean, invstd, dgamma, dbeta, inv_s,
-                                  static_cast<const int*>(nullptr), 0, pv.rows, pv.chunk, pv.tiles, pb.HW, pb.P)));
+                                  static_cast<const int*>(nullptr), 0, RowOrder{RowOrder::kIdentity, pv.rows, 0, 0},
+                                  pv.nchunks, pv.tiles, pb.HW, pb.P)));
         break;
     }
     return last_error();
@@ -640,7 +654,7 @@ int bns_set_tuning(const char* name, int value) {
         bool* bvalue;
     } knobs[] = {{"target_blocks", &g_target_blocks, nullptr},   {"min_chunk", &g_min_chunk, nullptr},
                  {"stat_target_blocks", &g_stat_target_blocks, nullptr}, {"stat_min_chunk", &g_stat_min_chunk, nullptr},
-                 {"pdl", nullptr, &g_pdl}};
+                 {"pdl", nullptr, &g_pdl},                       {"l2_order", nullptr, &g_l2_order}};
     for (const Knob& k : knobs) {
         if (std::strcmp(name, k.name) != 0) continue;
         if (k.ivalue) {

@@ -34,6 +34,25 @@ __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepco
 // Allow the next kernel of the stream to be scheduled once every block of this one got here.
 __device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
 
+// ------------------------------------------------------------------------------------ row order
+// Row chunks are interleaved: chunk ck of nchunks visits "virtual rows" ck, ck+nchunks, ck+2 nchunks, ...
+// so all blocks of a launch move through the tensor together and virtual row v is visited at about
+// the same time by every block.  RowOrder maps the virtual row to the sample it stands for, which
+// lets a kernel visit first the rows that the previous kernel left in L2, or leave for last the rows
+// that the next kernel will want there.  The order only permutes independent rows.
+struct RowOrder {
+    enum { kIdentity = 0, kRangeFirst = 1, kRangeLast = 2, kReversed = 3 };
+    int mode, rows, begin, count;  // [begin, begin+count): the range moved to the front or to the back
+    __device__ __forceinline__ int operator()(int v) const {
+        switch (mode) {
+        case kRangeFirst: return v < count ? begin + v : (v - count < begin ? v - count : v);
+        case kRangeLast: return v < begin ? v : (v < rows - count ? v + count : begin + v - (rows - count));
+        case kReversed: return rows - 1 - v;
+        default: return v;
+        }
+    }
+};
+
 // ------------------------------------------------------------------------------------ element types
 struct F32 {
     using storage = float;
@@ -352,35 +371,34 @@ __device__ __forceinline__ void fold_sums(const float* s_a, const float* s_b, co
 template <typename T, int V>
 __global__ void __launch_bounds__(kThreads)
 col_moments_kernel(const typename T::storage* __restrict__ x, const int* __restrict__ list, int begin, int count,
-                   int chunk, unsigned tiles, int HW, unsigned P, StatsSink S) {
+                   int nchunks, unsigned tiles, int HW, unsigned P, StatsSink S) {
     constexpr unsigned TP = kThreads * V;
     __shared__ float s_mean[TP];
     __shared__ float s_m2[TP];
     grid_dependency_wait();
     grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
-    const unsigned ck = blockIdx.x / tiles;
+    const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
-    const int i0 = ck * chunk, i1 = min(count, i0 + chunk);
-    const float cnt = static_cast<float>(i1 - i0);
+    const float cnt = static_cast<float>((count - ck + nchunks - 1) / nchunks);  // rows of this chunk
     float K[V], s1[V], s2[V];
 #pragma unroll
     for (int j = 0; j < V; ++j) K[j] = s1[j] = s2[j] = 0.f;
     if (p < P) {
         const typename T::storage* xp = x + p;
         {   // pivot: the first value of every position (its own deviation is zero)
-            int n = list ? list[i0] : begin + i0;
+            int n = list ? list[ck] : begin + ck;
             Vec<T, V> v;
             v.load(xp + static_cast<size_t>(n) * P);
 #pragma unroll
             for (int j = 0; j < V; ++j) K[j] = v.get(j);
         }
-        int i = i0 + 1;
-        for (; i + kUnroll <= i1; i += kUnroll) {
+        int i = ck + nchunks;
+        for (; i + (kUnroll - 1) * nchunks < count; i += kUnroll * nchunks) {
             Vec<T, V> v[kUnroll];
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
-                int n = list ? list[i + u] : begin + i + u;
+                int n = list ? list[i + u * nchunks] : begin + i + u * nchunks;
                 v[u].load(xp + static_cast<size_t>(n) * P);
             }
 #pragma unroll
@@ -392,7 +410,7 @@ col_moments_kernel(const typename T::storage* __restrict__ x, const int* __restr
                     s2[j] = fmaf(d, d, s2[j]);
                 }
         }
-        for (; i < i1; ++i) {
+        for (; i < count; i += nchunks) {
             int n = list ? list[i] : begin + i;
             Vec<T, V> v;
             v.load(xp + static_cast<size_t>(n) * P);
@@ -463,29 +481,28 @@ struct PatchThread {
 // Partial moments of the patch elements per (sample chunk, tile of compact positions, channel slot).
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
-patch_moments_kernel(const typename T::storage* __restrict__ x, PatchRule rule, int N, int C, int H, int W, int chunk,
+patch_moments_kernel(const typename T::storage* __restrict__ x, PatchRule rule, int N, int C, int H, int W, int nchunks,
                      unsigned tiles, StatsSink S, unsigned* status) {
     __shared__ float s_mean[kThreads];
     __shared__ float s_m2[kThreads];
     grid_dependency_wait();
     grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
-    const unsigned ck = blockIdx.x / tiles;
+    const int ck = static_cast<int>(blockIdx.x / tiles);
     const int PP = rule.ph * rule.pw;
     const unsigned Pc = static_cast<unsigned>(C) * PP;  // compact positions per sample
     const unsigned j = tile * kThreads + threadIdx.x;
     const size_t P = static_cast<size_t>(C) * H * W;
-    const int n0 = ck * chunk, n1 = min(N, n0 + chunk);
-    const float cnt = static_cast<float>(n1 - n0);
+    const float cnt = static_cast<float>((N - ck + nchunks - 1) / nchunks);  // samples of this chunk
     float K = 0.f, s1 = 0.f, s2 = 0.f;
     if (j < Pc) {
         const PatchThread me(j, rule, H, W);
-        K = to_float<T>(x[me.at(rule, n0, P, H, W, status)]);  // pivot: the first value
-        int n = n0 + 1;
-        for (; n + kUnroll <= n1; n += kUnroll) {
+        K = to_float<T>(x[me.at(rule, ck, P, H, W, status)]);  // pivot: the first value
+        int n = ck + nchunks;
+        for (; n + (kUnroll - 1) * nchunks < N; n += kUnroll * nchunks) {
             float v[kUnroll];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) v[u] = to_float<T>(x[me.at(rule, n + u, P, H, W, status)]);
+            for (int u = 0; u < kUnroll; ++u) v[u] = to_float<T>(x[me.at(rule, n + u * nchunks, P, H, W, status)]);
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 float d = v[u] - K;
@@ -493,7 +510,7 @@ patch_moments_kernel(const typename T::storage* __restrict__ x, PatchRule rule, 
                 s2 = fmaf(d, d, s2);
             }
         }
-        for (; n < n1; ++n) {
+        for (; n < N; n += nchunks) {
             float d = to_float<T>(x[me.at(rule, n, P, H, W, status)]) - K;
             s1 += d;
             s2 = fmaf(d, d, s2);
@@ -533,11 +550,11 @@ template <typename T, int V>
 __global__ void __launch_bounds__(kThreads)
 col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::storage* __restrict__ y,
                      const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
-                     const float* __restrict__ invstd, int rows, int chunk, unsigned tiles, int HW, unsigned P) {
+                     const float* __restrict__ invstd, RowOrder order, int nchunks, unsigned tiles, int HW, unsigned P) {
     grid_dependency_wait();
     grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
-    const unsigned ck = blockIdx.x / tiles;
+    const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
     if (p >= P) return;
     float a[V], b[V];
@@ -550,31 +567,31 @@ col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::stor
             b[j] = fmaf(-mean[c[j]], a[j], beta[c[j]]);
         }
     }
-    const int n0 = ck * chunk, n1 = min(rows, n0 + chunk);
-    const typename T::storage* xp = x + static_cast<size_t>(n0) * P + p;
-    typename T::storage* yp = y + static_cast<size_t>(n0) * P + p;
-    int n = n0;
-    for (; n + kUnroll <= n1; n += kUnroll) {
+    const typename T::storage* xp = x + p;
+    typename T::storage* yp = y + p;
+    int i = ck;
+    for (; i + (kUnroll - 1) * nchunks < order.rows; i += kUnroll * nchunks) {
         Vec<T, V> v[kUnroll];
+        int row[kUnroll];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) v[u].load(xp + static_cast<size_t>(u) * P);
+        for (int u = 0; u < kUnroll; ++u) {
+            row[u] = order(i + u * nchunks);
+            v[u].load(xp + static_cast<size_t>(row[u]) * P);
+        }
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
 #pragma unroll
             for (int j = 0; j < V; ++j) v[u].set(j, fmaf(a[j], v[u].get(j), b[j]));
-            v[u].store(yp + static_cast<size_t>(u) * P);
+            v[u].store(yp + static_cast<size_t>(row[u]) * P);
         }
-        xp += static_cast<size_t>(kUnroll) * P;
-        yp += static_cast<size_t>(kUnroll) * P;
     }
-    for (; n < n1; ++n) {
+    for (; i < order.rows; i += nchunks) {
+        const size_t off = static_cast<size_t>(order(i)) * P;
         Vec<T, V> v;
-        v.load(xp);
+        v.load(xp + off);
 #pragma unroll
         for (int j = 0; j < V; ++j) v.set(j, fmaf(a[j], v.get(j), b[j]));
-        v.store(yp);
-        xp += P;
-        yp += P;
+        v.store(yp + off);
     }
 }
 
@@ -585,7 +602,7 @@ template <typename T, int V, bool WRITE_DX>
 __global__ void __launch_bounds__(kThreads)
 col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
                       typename T::storage* __restrict__ dx, const float* __restrict__ gamma,
-                      const float* __restrict__ mean, const float* __restrict__ invstd, int rows, int chunk,
+                      const float* __restrict__ mean, const float* __restrict__ invstd, RowOrder order, int nchunks,
                       unsigned tiles, int HW, unsigned P, bool virtual_pass, GradSink G) {
     constexpr unsigned TP = kThreads * V;
     __shared__ float s_dy[TP];
@@ -593,7 +610,7 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
     grid_dependency_wait();
     grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
-    const unsigned ck = blockIdx.x / tiles;
+    const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
     float acc_dy[V], acc_dyxc[V];
 #pragma unroll
@@ -609,18 +626,18 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
                 a[j] = WRITE_DX ? gamma[c[j]] * invstd[c[j]] : 0.f;
             }
         }
-        const int n0 = ck * chunk, n1 = min(rows, n0 + chunk);
-        const size_t base = static_cast<size_t>(n0) * P + p;
-        const typename T::storage* xp = x + base;
-        const typename T::storage* gp = dy + base;
-        typename T::storage* op = WRITE_DX ? dx + base : nullptr;
-        int n = n0;
-        for (; n + kUnroll <= n1; n += kUnroll) {
+        const typename T::storage* xp = x + p;
+        const typename T::storage* gp = dy + p;
+        typename T::storage* op = WRITE_DX ? dx + p : nullptr;
+        int i = ck;
+        for (; i + (kUnroll - 1) * nchunks < order.rows; i += kUnroll * nchunks) {
             Vec<T, V> vx[kUnroll], vg[kUnroll];
+            int row[kUnroll];
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
-                vx[u].load(xp + static_cast<size_t>(u) * P);
-                vg[u].load(gp + static_cast<size_t>(u) * P);
+                row[u] = order(i + u * nchunks);
+                vx[u].load(xp + static_cast<size_t>(row[u]) * P);
+                vg[u].load(gp + static_cast<size_t>(row[u]) * P);
             }
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
@@ -631,16 +648,14 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
                     acc_dyxc[j] = fmaf(g, vx[u].get(j) - mu[j], acc_dyxc[j]);
                     if (WRITE_DX) vg[u].set(j, a[j] * g);
                 }
-                if (WRITE_DX) vg[u].store(op + static_cast<size_t>(u) * P);
+                if (WRITE_DX) vg[u].store(op + static_cast<size_t>(row[u]) * P);
             }
-            xp += static_cast<size_t>(kUnroll) * P;
-            gp += static_cast<size_t>(kUnroll) * P;
-            if (WRITE_DX) op += static_cast<size_t>(kUnroll) * P;
         }
-        for (; n < n1; ++n) {
+        for (; i < order.rows; i += nchunks) {
+            const size_t off = static_cast<size_t>(order(i)) * P;
             Vec<T, V> vx, vg;
-            vx.load(xp);
-            vg.load(gp);
+            vx.load(xp + off);
+            vg.load(gp + off);
 #pragma unroll
             for (int j = 0; j < V; ++j) {
                 float g = vg.get(j);
@@ -648,12 +663,7 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
                 acc_dyxc[j] = fmaf(g, vx.get(j) - mu[j], acc_dyxc[j]);
                 if (WRITE_DX) vg.set(j, a[j] * g);
             }
-            if (WRITE_DX) {
-                vg.store(op);
-                op += P;
-            }
-            xp += P;
-            gp += P;
+            if (WRITE_DX) vg.store(op + off);
         }
     }
 #pragma unroll
@@ -690,12 +700,12 @@ __global__ void __launch_bounds__(kThreads)
 col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
                  typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
                  const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
-                 float inv_s, const int* __restrict__ list, int begin, int count, int chunk, unsigned tiles, int HW,
-                 unsigned P) {
+                 float inv_s, const int* __restrict__ list, int begin, RowOrder order, int nchunks, unsigned tiles,
+                 int HW, unsigned P) {
     grid_dependency_wait();
     grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
-    const unsigned ck = blockIdx.x / tiles;
+    const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
     if (p >= P) return;
     FixCoef k[V];
@@ -705,17 +715,16 @@ col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::st
 #pragma unroll
         for (int j = 0; j < V; ++j) k[j] = fix_coef(gamma[c[j]], mean[c[j]], invstd[c[j]], dgamma[c[j]], dbeta[c[j]], inv_s);
     }
-    const int i0 = ck * chunk, i1 = min(count, i0 + chunk);
-    int i = i0;
-    for (; i + kUnroll <= i1; i += kUnroll) {
+    int i = ck;
+    for (; i + (kUnroll - 1) * nchunks < order.rows; i += kUnroll * nchunks) {
         Vec<T, V> vx[kUnroll], vg[kUnroll];
-        size_t off[kUnroll];
+        int row[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-            int n = list ? list[i + u] : begin + i + u;
-            off[u] = static_cast<size_t>(n) * P + p;
-            vx[u].load(x + off[u]);
-            if (dy) vg[u].load(dy + off[u]);
+            int v = order(i + u * nchunks);
+            row[u] = list ? list[v] : begin + v;
+            vx[u].load(x + static_cast<size_t>(row[u]) * P + p);
+            if (dy) vg[u].load(dy + static_cast<size_t>(row[u]) * P + p);
         }
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
@@ -724,11 +733,12 @@ col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::st
                 float g = dy ? vg[u].get(j) : 0.f;
                 vg[u].set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (vx[u].get(j) - k[j].mu));
             }
-            vg[u].store(dx + off[u]);
+            vg[u].store(dx + static_cast<size_t>(row[u]) * P + p);
         }
     }
-    for (; i < i1; ++i) {
-        int n = list ? list[i] : begin + i;
+    for (; i < order.rows; i += nchunks) {
+        int v = order(i);
+        int n = list ? list[v] : begin + v;
         size_t off = static_cast<size_t>(n) * P + p;
         Vec<T, V> vx, vg;
         vx.load(x + off);
@@ -748,32 +758,31 @@ __global__ void __launch_bounds__(kThreads)
 patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
                    typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
                    const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
-                   float inv_s, PatchRule rule, int N, int C, int H, int W, int chunk, unsigned tiles,
+                   float inv_s, PatchRule rule, int N, int C, int H, int W, int nchunks, unsigned tiles,
                    unsigned* status) {
     grid_dependency_wait();
     grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
-    const unsigned ck = blockIdx.x / tiles;
+    const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned j = tile * kThreads + threadIdx.x;
     if (j >= static_cast<unsigned>(C) * rule.ph * rule.pw) return;
     const PatchThread me(j, rule, H, W);
     const size_t P = static_cast<size_t>(C) * H * W;
     const FixCoef k = fix_coef(gamma[me.c], mean[me.c], invstd[me.c], dgamma[me.c], dbeta[me.c], inv_s);
-    const int n0 = ck * chunk, n1 = min(N, n0 + chunk);
-    int n = n0;
-    for (; n + kUnroll <= n1; n += kUnroll) {
+    int n = ck;
+    for (; n + (kUnroll - 1) * nchunks < N; n += kUnroll * nchunks) {
         size_t at[kUnroll];
         float g[kUnroll], xv[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-            at[u] = me.at(rule, n + u, P, H, W, status);
+            at[u] = me.at(rule, n + u * nchunks, P, H, W, status);
             g[u] = to_float<T>(dy[at[u]]);
             xv[u] = to_float<T>(x[at[u]]);
         }
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) dx[at[u]] = from_float<T>(fmaf(k.a, g[u], -k.A) - k.Q * (xv[u] - k.mu));
     }
-    for (; n < n1; ++n) {
+    for (; n < N; n += nchunks) {
         size_t at = me.at(rule, n, P, H, W, status);
         float g = to_float<T>(dy[at]), xv = to_float<T>(x[at]);
         dx[at] = from_float<T>(fmaf(k.a, g, -k.A) - k.Q * (xv - k.mu));

@@ -214,5 +214,5 @@ def test_other_grid_shapes_still_match_the_oracle(target):
             case = make_case(70, 12, 33, 31, rule, seed=86, **kw)
             compare(case, run_gpu(case))
     finally:
-        bns.set_tuning("target_blocks", 148 * 8)
+        bns.set_tuning("target_blocks", 148 * 32)
         bns.set_tuning("stat_target_blocks", 148 * 8)
