@@ -130,6 +130,36 @@ bns_status bns_full_bn(const bns_shape* shape, const void* x, const float* gamma
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * bns_forward for callers that cannot provide scratch memory.  (The paper has no counterpart; this
+ * is a packaging variant of bns_forward: same kernels, same results.)
+ *
+ * Some hosts of this library are not allowed to allocate on the device: a plug-in inside an
+ * inference server or framework that has handed all device memory to its own pool, code that runs
+ * where cudaMalloc is forbidden because it synchronises the whole device under other tenants'
+ * streams, or a component that ships with a fixed memory map.  Such a caller has its input and
+ * output tensors (the host application gave them to it) but no workspace.  This entry point uses
+ * scratch that is built into the library image instead: a 4 MiB array in device memory
+ * (bns_static_workspace_bytes()), which every GPU that loads the library holds until the process
+ * exits.  It calls no cudaMalloc/cudaFree and no allocating routine of any library.
+ *
+ *  - Arguments and results are those of bns_forward, minus the workspace pair.
+ *  - A shape/rule whose bns_workspace_bytes() exceeds bns_static_workspace_bytes() is rejected with
+ *    BNS_ERR_WORKSPACE before anything is launched (the ResNet-50 layers at N=256 need up to 2.6 MB).
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *    that device current) and keeps it; make that first call before any stream capture begins.
+ *  - All calls on a device share the one array, which keeps whatever the previous call left in it.
+ *    Nothing in it needs to start at zero (the status word is cleared by the call when it is used),
+ *    but two calls that overlap in time on the same GPU - different streams, or different host
+ *    threads - would overwrite each other's partial sums: run them one after the other.
+ *  - bns_workspace_status() cannot read this scratch: device-resident patch offsets are still
+ *    clamped into range, but the flag is not retrievable through this entry point.
+ */
+size_t bns_static_workspace_bytes(void);
+bns_status bns_forward_static(const bns_shape* shape, const void* x, const float* gamma, const float* beta,
+                              float eps, const bns_sampling* sampling, void* y, float* mean, float* invstd,
+                              void* cuda_stream);
+
+/*
  * Forward and backward of one layer with HOST buffers for the large tensors: copies x and dy to
  * the device, runs bns_forward and bns_backward, copies y, dx, mean, invstd, dgamma, dbeta back.
  * x, dy, y, dx, gamma, beta and the six outputs are HOST pointers (pinned memory lets the copies

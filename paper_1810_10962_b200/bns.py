@@ -28,7 +28,7 @@ KERNEL_KINDS = 9
  KERNEL_FINALIZE_BWD, KERNEL_COL_FIXUP, KERNEL_PATCH_FIXUP, KERNEL_MASK) = range(KERNEL_KINDS)
 
 EXPORTS = [
-    "bns_workspace_bytes", "bns_forward", "bns_backward", "bns_full_bn", "bns_host_arena_bytes",
+    "bns_workspace_bytes", "bns_forward", "bns_forward_static", "bns_static_workspace_bytes", "bns_backward", "bns_full_bn", "bns_host_arena_bytes",
     "bns_forward_backward_host", "bns_debug_selection_mask", "bns_workspace_status", "bns_status_string",
     "bns_launch_count", "bns_launch_count_reset", "bns_profile_enable", "bns_profile_read", "bns_kernel_name",
     "bns_set_tuning",
@@ -80,6 +80,10 @@ def load():
     lib.bns_workspace_bytes.argtypes = [shp, smp]
     lib.bns_forward.restype = ctypes.c_int
     lib.bns_forward.argtypes = [shp, vp, vp, vp, fl, smp, vp, vp, vp, vp, sz, vp]
+    lib.bns_forward_static.restype = ctypes.c_int
+    lib.bns_forward_static.argtypes = [shp, vp, vp, vp, fl, smp, vp, vp, vp, vp]
+    lib.bns_static_workspace_bytes.restype = sz
+    lib.bns_static_workspace_bytes.argtypes = []
     lib.bns_backward.restype = ctypes.c_int
     lib.bns_backward.argtypes = [shp, vp, vp, vp, vp, vp, smp, vp, vp, vp, vp, sz, vp]
     lib.bns_full_bn.restype = ctypes.c_int
@@ -245,6 +249,22 @@ def forward(x, gamma, beta, eps, sampling: Sampling, y=None, mean=None, invstd=N
     st = load().bns_forward(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), ctypes.byref(sp),
                             _dev(y), _vec(mean, C), _vec(invstd, C), wp, wn, _stream())
     _check(st, "bns_forward")
+    return y, mean, invstd
+
+
+def static_workspace_bytes() -> int:
+    return int(load().bns_static_workspace_bytes())
+
+
+def forward_static(x, gamma, beta, eps, sampling: Sampling, y, mean, invstd):
+    """bns_forward_static: the forward for callers that may not allocate device memory.  The caller
+    passes every tensor, outputs included; the scratch is the array built into the library, shared by
+    all calls on the device (so do not overlap two of them).  Returns (y, mean, invstd)."""
+    sh, sp = _shape(x), sampling._c()
+    C = x.shape[1]
+    st = load().bns_forward_static(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps),
+                                   ctypes.byref(sp), _dev(y), _vec(mean, C), _vec(invstd, C), _stream())
+    _check(st, "bns_forward_static")
     return y, mean, invstd
 
 

@@ -683,4 +683,50 @@ const char* bns_kernel_name(int kernel_kind) {
     return "unknown";
 }
 
+// ---------------------------------------------------------------------------------------- no-allocation forward
+// Scratch for bns_forward_static: a fixed array in device memory that is part of the loaded library
+// image, so a caller that has no way to obtain device memory of its own can still run the forward.
+// The name below is only a host-side handle; the address the kernels need is looked up per device.
+#define BNS_STATIC_WORKSPACE_BYTES (4u << 20)
+static __device__ __align__(256) unsigned char g_static_workspace[BNS_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_workspace_address[kMaxDevices] = {};  // resolved by the first call made on each device
+
+// Device address of the static scratch on the device that is current now.
+bns_status static_workspace_address(void** address) {
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return BNS_ERR_CUDA;
+    if (device < 0 || device >= kMaxDevices) return BNS_ERR_CUDA;
+    if (!g_static_workspace_address[device]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return BNS_ERR_CUDA;
+        g_static_workspace_address[device] = p;
+    }
+    *address = g_static_workspace_address[device];
+    return BNS_OK;
+}
+}  // namespace
+
+size_t bns_static_workspace_bytes(void) { return BNS_STATIC_WORKSPACE_BYTES; }
+
+bns_status bns_forward_static(const bns_shape* shape, const void* x, const float* gamma, const float* beta, float eps,
+                              const bns_sampling* sampling, void* y, float* mean, float* invstd, void* cuda_stream) {
+    Problem pb;
+    bns_status st = make_problem(shape, sampling, pb);
+    if (st != BNS_OK) return st;
+    if (!x || !gamma || !beta || !y || !mean || !invstd) return BNS_ERR_NULL;
+    if (!(eps > 0.f)) return BNS_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(y)) return BNS_ERR_ALIGN;
+    if (pb.total > BNS_STATIC_WORKSPACE_BYTES) return BNS_ERR_WORKSPACE;  // needs more scratch than is built in
+    void* workspace = nullptr;
+    st = static_workspace_address(&workspace);
+    if (st != BNS_OK) return st;
+    // Nothing in the scratch has to start at zero except the status word, which forward_impl clears itself
+    // whenever a kernel may set it; every partial sum is written before it is read.
+    return forward_impl(pb, sampling, x, gamma, beta, eps, y, mean, invstd, workspace,
+                        static_cast<cudaStream_t>(cuda_stream));
+}
+
 }  // extern "C"
