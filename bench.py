@@ -242,6 +242,21 @@ class DeviceLayer:
                    workspace=self.ws)
 
 
+def slowest_rank_ms(torch, dist, ms, world, device):
+    """Per-step time of the slowest rank (the ranks are independent replicas; the job is as slow as
+    its slowest one).  `dist` is an initialised torch.distributed or None when world == 1."""
+    if world <= 1:
+        return float(ms)
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbps(step_bytes, world, ms):
+    """Bytes moved by all replicas in one step over the slowest rank's step time."""
+    return world * step_bytes / (ms * 1e-3) / 1e9
+
+
 def time_steps(torch, dist, run_step, steps, warmup, device_index, world):
     """W warm-up steps, then exactly K steps between CUDA events on the current stream, bracketed by a
     barrier and a device synchronise on both sides.  Returns (ms per step: max over ranks, clocks)."""
@@ -262,10 +277,8 @@ def time_steps(torch, dist, run_step, steps, warmup, device_index, world):
     clocks = sampler.stop()
     ms = start.elapsed_time(stop) / steps
     if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = slowest_rank_ms(torch, dist, ms, world, "cuda")
         dist.barrier()
-        ms = float(t.item())
     torch.cuda.synchronize()
     return ms, clocks
 
@@ -327,7 +340,7 @@ def run_ours(args):
     bns.profile_enable(False)
     # ---- the same K steps with the library's per-kernel events off: the reported value
     ms_plain, clocks_plain = time_steps(torch, dist, step, args.steps, args.warmup, local, world)
-    value = world * step_bytes / (ms_plain * 1e-3) / 1e9
+    value = whole_job_gbps(step_bytes, world, ms_plain)
     peak, peak_source = measured_hbm_peak()
 
     # ---- per-layer numbers and the full-BN comparison (same protocol, each layer alone)
