@@ -551,11 +551,26 @@ __global__ void __launch_bounds__(kThreads)
 col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::storage* __restrict__ y,
                      const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
                      const float* __restrict__ invstd, RowOrder order, int nchunks, unsigned tiles, int HW, unsigned P) {
-    grid_dependency_wait();
-    grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
     const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
+    const typename T::storage* xp = x + p;
+    typename T::storage* yp = y + p;
+    // x is an input of the whole call, so the first rows can be requested before the statistics
+    // kernels ahead of this one have finished; only mean / invstd have to wait for them.
+    int i = ck;
+    const bool head = p < P && i + (kUnroll - 1) * nchunks < order.rows;
+    Vec<T, V> v[kUnroll];
+    int row[kUnroll];
+    if (head) {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            row[u] = order(i + u * nchunks);
+            v[u].load(xp + static_cast<size_t>(row[u]) * P);
+        }
+    }
+    grid_dependency_wait();
+    grid_dependency_launch();
     if (p >= P) return;
     float a[V], b[V];
     {
@@ -567,12 +582,16 @@ col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::stor
             b[j] = fmaf(-mean[c[j]], a[j], beta[c[j]]);
         }
     }
-    const typename T::storage* xp = x + p;
-    typename T::storage* yp = y + p;
-    int i = ck;
+    if (head) {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+#pragma unroll
+            for (int j = 0; j < V; ++j) v[u].set(j, fmaf(a[j], v[u].get(j), b[j]));
+            v[u].store(yp + static_cast<size_t>(row[u]) * P);
+        }
+        i += kUnroll * nchunks;
+    }
     for (; i + (kUnroll - 1) * nchunks < order.rows; i += kUnroll * nchunks) {
-        Vec<T, V> v[kUnroll];
-        int row[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
             row[u] = order(i + u * nchunks);
@@ -587,11 +606,11 @@ col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::stor
     }
     for (; i < order.rows; i += nchunks) {
         const size_t off = static_cast<size_t>(order(i)) * P;
-        Vec<T, V> v;
-        v.load(xp + off);
+        Vec<T, V> w;
+        w.load(xp + off);
 #pragma unroll
-        for (int j = 0; j < V; ++j) v.set(j, fmaf(a[j], v.get(j), b[j]));
-        v.store(yp + off);
+        for (int j = 0; j < V; ++j) w.set(j, fmaf(a[j], w.get(j), b[j]));
+        w.store(yp + off);
     }
 }
 
