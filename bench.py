@@ -230,16 +230,62 @@ class DeviceLayer:
             xv = torch.from_numpy(host["xv"]).cuda()
             self.sp = bns.Sampling.virtual(xv, yv=torch.empty_like(xv), dyv=None, dxv=torch.empty_like(xv))
         self.ws = bns.new_workspace(x, self.sp)
+        # argument marshalling done once per buffer set; a step is then two C calls per layer
+        self.calls = [bns.Prepared(sx, sdy, self.gamma, self.beta, EPS, self.sp, sy, sdx, self.mean, self.invstd,
+                                   self.dgamma, self.dbeta, self.ws, full_bn_entry=self.full)
+                      for sx, sdy, sy, sdx in self.sets]
 
     def step(self, i):
-        x, dy, y, dx = self.sets[i % len(self.sets)]
-        b = self.bns
-        if self.full:
-            b.full_bn(x, self.gamma, self.beta, EPS, y=y, mean=self.mean, invstd=self.invstd, workspace=self.ws)
-        else:
-            b.forward(x, self.gamma, self.beta, EPS, self.sp, y=y, mean=self.mean, invstd=self.invstd, workspace=self.ws)
-        b.backward(x, dy, self.gamma, self.mean, self.invstd, self.sp, dx=dx, dgamma=self.dgamma, dbeta=self.dbeta,
-                   workspace=self.ws)
+        call = self.calls[i % len(self.calls)]
+        call.forward()
+        call.backward()
+
+
+def capture_steps(torch, step, sets):
+    """Captures `sets` consecutive steps (one per rotating buffer set) into a CUDA graph, so that the
+    timed loop replays kernels without per-call host work.  Returns None if capture is not possible."""
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(sets):
+                step(i)                      # warm up on the capture stream
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(sets):
+                step(i)
+        graph.replay()
+        torch.cuda.synchronize()
+        return graph
+    except Exception as exc:                 # keep measuring eagerly
+        print(f"bench: CUDA graph capture failed ({exc}); timing eager launches", file=sys.stderr)
+        torch.cuda.synchronize()
+        return None
+
+
+class GraphedSteps:
+    """Step function for time_steps: a loop of n steps is run as n // sets graph replays (each replay is
+    `sets` steps) plus n % sets eager steps, so exactly n steps execute."""
+
+    def __init__(self, graph, step, sets):
+        self.graph, self.step, self.sets = graph, step, sets
+        self.remaining = self.covered = 0
+
+    def begin(self, n):
+        self.remaining, self.covered = n, 0
+
+    def __call__(self, i):
+        if self.covered == 0:
+            if self.remaining >= self.sets:
+                self.graph.replay()
+                self.covered = self.sets
+            else:
+                self.step(i)
+                self.covered = 1
+        self.covered -= 1
+        self.remaining -= 1
 
 
 def slowest_rank_ms(torch, dist, ms, world, device):
@@ -260,6 +306,8 @@ def whole_job_gbps(step_bytes, world, ms):
 def time_steps(torch, dist, run_step, steps, warmup, device_index, world):
     """W warm-up steps, then exactly K steps between CUDA events on the current stream, bracketed by a
     barrier and a device synchronise on both sides.  Returns (ms per step: max over ranks, clocks)."""
+    begin = getattr(run_step, "begin", lambda n: None)
+    begin(warmup)
     for i in range(warmup):
         run_step(i)
     torch.cuda.synchronize()
@@ -269,6 +317,7 @@ def time_steps(torch, dist, run_step, steps, warmup, device_index, world):
     sampler = ClockSampler(device_index)
     sampler.start()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    begin(steps)
     start.record()
     for i in range(steps):
         run_step(warmup + i)
@@ -339,24 +388,29 @@ def run_ours(args):
             kernel_times[bns.kernel_name(kind)] = {"launches": n, "total_ms": round(tot, 4), "avg_us": round(1e3 * tot / n, 3)}
     bns.profile_enable(False)
     # ---- the same K steps with the library's per-kernel events off: the reported value
-    ms_plain, clocks_plain = time_steps(torch, dist, step, args.steps, args.warmup, local, world)
+    def runner(fn):
+        g = capture_steps(torch, fn, sets) if args.graph else None
+        return (GraphedSteps(g, fn, sets) if g else fn), g is not None
+
+    run, graphed = runner(step)
+    ms_plain, clocks_plain = time_steps(torch, dist, run, args.steps, args.warmup, local, world)
     value = whole_job_gbps(step_bytes, world, ms_plain)
     peak, peak_source = measured_hbm_peak()
 
     # ---- per-layer numbers and the full-BN comparison (same protocol, each layer alone)
     per_layer = {}
     for d in dev:
-        lms, _ = time_steps(torch, dist, d.step, args.steps, args.warmup, local, world)
+        lms, _ = time_steps(torch, dist, runner(d.step)[0], args.steps, args.warmup, local, world)
         per_layer[d.layer.name] = {"ms": round(lms, 5), "gbps": round(d.layer.algorithmic_bytes() / lms / 1e6, 1),
                                    "algorithmic_bytes": d.layer.algorithmic_bytes(), "count": d.layer.count}
     full_info = None
     if full:
-        fms, _ = time_steps(torch, dist, full_step, args.steps, args.warmup, local, world)
+        fms, _ = time_steps(torch, dist, runner(full_step)[0], args.steps, args.warmup, local, world)
         fbytes = sum(l.count * (8 * l.elems * l.ebytes + 32 * l.C) for l in layers)
         full_info = {"ms_per_step": round(fms, 5), "gbps": round(fbytes / fms / 1e6, 1), "algorithmic_bytes": fbytes,
                      "speedup_sampled_vs_full": round(fms / ms_plain, 4)}
         for d in full:
-            lms, _ = time_steps(torch, dist, d.step, args.steps, args.warmup, local, world)
+            lms, _ = time_steps(torch, dist, runner(d.step)[0], args.steps, args.warmup, local, world)
             per_layer[d.layer.name]["full_bn_ms"] = round(lms, 5)
             per_layer[d.layer.name]["speedup_vs_full_bn"] = round(lms / per_layer[d.layer.name]["ms"], 4)
 
@@ -394,6 +448,7 @@ def run_ours(args):
                        "layers": [f"{l.name}:{l.N}x{l.C}x{l.H}x{l.W}:{l.dtype}:x{l.count}" for l in layers],
                        "step": "forward+backward of every layer", "algorithmic_bytes_per_step": step_bytes,
                        "cache": f"inputs larger than L2; {sets} buffer sets rotated", "replicas": world,
+                       "launch": f"CUDA graph replay, {sets} steps per graph" if graphed else "eager launches",
                        "tuning": args.tune},
             "frac_of_hbm_peak": round(value / world / peak, 4), "hbm_peak_gbs": peak, "hbm_peak_source": peak_source,
             "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
@@ -545,6 +600,8 @@ def main():
     ap.add_argument("--tune", action="append", default=[], metavar="NAME=VALUE",
                     help="launch-shape knob of the library (bns_set_tuning), e.g. --tune pdl=0")
     ap.add_argument("--no-full-bn", dest="full_bn", action="store_false", help="skip the full-BN comparison")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="time eager launches instead of replaying a CUDA graph of the step")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the oracle baseline (0 = skip)")

@@ -198,7 +198,9 @@ typedef enum {
     BNS_KERNEL_COL_FIXUP = 6,     /* gradient with the statistics terms over whole samples      */
     BNS_KERNEL_PATCH_FIXUP = 7,   /* the same over patches                                      */
     BNS_KERNEL_MASK = 8,
-    BNS_KERNEL_KINDS = 9
+    BNS_KERNEL_DIRECT_MOMENTS = 9, /* statistics of a small sampled set, one block per channel    */
+    BNS_KERNEL_DIRECT_FIXUP = 10,  /* backward sums combined + statistics terms, small sampled set */
+    BNS_KERNEL_KINDS = 11
 } bns_kernel_kind;
 
 /* Number of kernels this library has launched in this process since load (or since reset). */
@@ -214,7 +216,9 @@ const char* bns_kernel_name(int kernel_kind);
 /* Launch-shape knobs (process-wide; change them only while no call is in flight, and recompute
  * bns_workspace_bytes afterwards).  "target_blocks" / "min_chunk": blocks per launch and least rows
  * per block of the streaming kernels; "stat_target_blocks" / "stat_min_chunk": the same for the
- * statistics kernels; "pdl": 0/1 programmatic dependent launch; "l2_order": 0/1 visit rows in an
+ * statistics kernels; "direct_max": sampled elements per channel up to which one block per channel computes the
+ * statistics (and, in the backward, combines the sums and applies the statistics terms) without
+ * partial sums, 0 = never; "pdl": 0/1 programmatic dependent launch; "l2_order": 0/1 visit rows in an
  * order that lets a kernel find in L2 what the previous one read.  Returns BNS_OK,
  * BNS_ERR_RULE for an unknown name or BNS_ERR_SHAPE for a value < 1. */
 int bns_set_tuning(const char* name, int value);

@@ -23,9 +23,10 @@ RULE_FULL, RULE_BATCH, RULE_FEATURE, RULE_VIRTUAL = 0, 1, 2, 3
 OFF_SHARED, OFF_PER_SAMPLE, OFF_PER_MAP = 0, 1, 2
 FLAG_BAD_OFFSET = 1
 
-KERNEL_KINDS = 9
+KERNEL_KINDS = 11
 (KERNEL_COL_MOMENTS, KERNEL_PATCH_MOMENTS, KERNEL_FINALIZE_STATS, KERNEL_NORMALIZE, KERNEL_BWD_REDUCE,
- KERNEL_FINALIZE_BWD, KERNEL_COL_FIXUP, KERNEL_PATCH_FIXUP, KERNEL_MASK) = range(KERNEL_KINDS)
+ KERNEL_FINALIZE_BWD, KERNEL_COL_FIXUP, KERNEL_PATCH_FIXUP, KERNEL_MASK, KERNEL_DIRECT_MOMENTS,
+ KERNEL_DIRECT_FIXUP) = range(KERNEL_KINDS)
 
 EXPORTS = [
     "bns_workspace_bytes", "bns_forward", "bns_forward_static", "bns_static_workspace_bytes", "bns_backward", "bns_full_bn", "bns_host_arena_bytes",
@@ -312,6 +313,51 @@ def workspace_status(workspace: torch.Tensor) -> int:
     flags = ctypes.c_uint32(0)
     _check(load().bns_workspace_status(workspace.data_ptr(), ctypes.byref(flags), _stream()), "bns_workspace_status")
     return int(flags.value)
+
+
+class Prepared:
+    """One layer's forward/backward with the argument marshalling done once.
+
+    For a training loop that calls the same layer on the same buffers every step: the ctypes structures
+    and raw pointers are built here, and forward() / backward() only make the C call (on the CUDA stream
+    that is current at call time).  The tensors are kept alive by this object."""
+
+    def __init__(self, x, dy, gamma, beta, eps, sampling: Sampling, y, dx, mean, invstd, dgamma, dbeta, workspace,
+                 full_bn_entry=False):
+        C = x.shape[1]
+        if dy.shape != x.shape or dy.dtype != x.dtype:
+            raise TypeError("dy must match x")
+        self._keep = (x, dy, gamma, beta, sampling, y, dx, mean, invstd, dgamma, dbeta, workspace)
+        self._lib = load()
+        self._sh, self._sp = _shape(x), sampling._c()
+        self._eps = float(eps)
+        self._full = bool(full_bn_entry)
+        self._x, self._dy, self._y, self._dx = _dev(x), _dev(dy), _dev(y), _dev(dx)
+        self._gamma, self._beta = _vec(gamma, C), _vec(beta, C)
+        self._mean, self._invstd = _vec(mean, C), _vec(invstd, C)
+        self._dgamma, self._dbeta = _vec(dgamma, C), _vec(dbeta, C)
+        self._ws, self._wn = workspace.data_ptr(), workspace.numel()
+        if self._wn < workspace_bytes(x, sampling):
+            raise BnsError(-7, "workspace too small")
+
+    def forward(self):
+        stream = torch.cuda.current_stream().cuda_stream
+        if self._full:
+            st = self._lib.bns_full_bn(ctypes.byref(self._sh), self._x, self._gamma, self._beta, self._eps, self._y,
+                                       self._mean, self._invstd, self._ws, self._wn, stream)
+        else:
+            st = self._lib.bns_forward(ctypes.byref(self._sh), self._x, self._gamma, self._beta, self._eps,
+                                       ctypes.byref(self._sp), self._y, self._mean, self._invstd, self._ws, self._wn,
+                                       stream)
+        if st != OK:
+            raise BnsError(st, "bns_forward")
+
+    def backward(self):
+        st = self._lib.bns_backward(ctypes.byref(self._sh), self._x, self._dy, self._gamma, self._mean, self._invstd,
+                                    ctypes.byref(self._sp), self._dx, self._dgamma, self._dbeta, self._ws, self._wn,
+                                    torch.cuda.current_stream().cuda_stream)
+        if st != OK:
+            raise BnsError(st, "bns_backward")
 
 
 # ----------------------------------------------------------------------------- host-buffer step

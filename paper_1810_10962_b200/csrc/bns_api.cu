@@ -279,7 +279,8 @@ bns_status clear_status(const Problem& pb, void* ws, cudaStream_t stream, unsign
 
 // ------------------------------------------------------------------------------------ launches
 bool g_pdl = true;    // ask for programmatic dependent launch (blocks may be scheduled while the previous kernel drains)
-bool g_l2_order = true;  // order rows so that a kernel re-reads what the previous one left in L2
+bool g_l2_order = true;
+int g_direct_max = 8192;  // sampled elements per channel up to which one block per channel handles the sampled set  // order rows so that a kernel re-reads what the previous one left in L2
 
 template <typename... KArgs, typename... Args>
 void launch(int kind, void (*kernel)(KArgs...), unsigned grid, cudaStream_t s, Args&&... args) {
@@ -339,9 +340,41 @@ typename T::storage* out(void* p) {
 
 unsigned warp_per_channel_grid(int C) { return static_cast<unsigned>((C + kThreads / 32 - 1) / (kThreads / 32)); }
 
+// Small sampled sets are handled by one block per channel (no partials, no finalize launch).
+bool small_sampled_set(const Problem& pb) { return pb.rule != BNS_RULE_FULL && pb.s <= static_cast<double>(g_direct_max); }
+
+SampleSet sample_set(const Problem& pb, const int* list) {
+    SampleSet set{};
+    set.patches = pb.rule == BNS_RULE_FEATURE;
+    set.list = list;
+    set.begin = pb.rule == BNS_RULE_BATCH ? pb.begin : 0;
+    set.rows = pb.count;
+    set.patch = pb.patch;
+    set.N = pb.N;
+    set.C = pb.C;
+    set.H = pb.H;
+    set.W = pb.W;
+    set.s = static_cast<int>(pb.s);
+    return set;
+}
+
 // Statistics of the rule's sampled set into mean / invstd: partial moments, then one warp per channel.
 bns_status run_statistics(const Problem& pb, const bns_sampling* sp, const void* x, float eps, float* mean,
                           float* invstd, void* ws, cudaStream_t stream) {
+    if (small_sampled_set(pb)) {
+        unsigned* status;
+        bns_status st = clear_status(pb, ws, stream, &status);
+        if (st != BNS_OK) return st;
+        const int* list = nullptr;
+        st = stage_list(pb, sp, ws, stream, &list);
+        if (st != BNS_OK) return st;
+        const SampleSet set = sample_set(pb, list);
+        const void* data = pb.rule == BNS_RULE_VIRTUAL ? sp->xv : x;
+        const int dt = pb.rule == BNS_RULE_VIRTUAL ? sp->xv_dtype : pb.dtype;
+        BNS_BY_TYPE(dt, (launch(BNS_KERNEL_DIRECT_MOMENTS, direct_moments_kernel<T>, static_cast<unsigned>(pb.C), stream,
+                                in<T>(data), set, eps, mean, invstd, status)));
+        return last_error();
+    }
     StatsSink sink{ws_at<float4>(ws, pb.off_stats), PartialLayout{}, static_cast<float>(1.0 / pb.s), eps, mean, invstd};
     int span = pb.HW;  // positions per channel in the producer's position space
     if (pb.rule == BNS_RULE_FEATURE) {
@@ -424,6 +457,26 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
                               in<T>(sp->dyv), out<T>(nullptr), gamma, mean, invstd,
                               RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P, true,
                               sink)));
+    if (small_sampled_set(pb)) {
+        // one block per channel combines the channel's sums and applies the statistics terms to its sampled set
+        unsigned* status;
+        bns_status st = clear_status(pb, ws, stream, &status);
+        if (st != BNS_OK) return st;
+        const int* list = nullptr;
+        st = stage_list(pb, sp, ws, stream, &list);
+        if (st != BNS_OK) return st;
+        const SampleSet set = sample_set(pb, list);
+        if (pb.rule == BNS_RULE_VIRTUAL)
+            BNS_BY_TYPE(sp->xv_dtype,
+                        (launch(BNS_KERNEL_DIRECT_FIXUP, direct_finalize_fixup_kernel<T>, static_cast<unsigned>(pb.C),
+                                stream, in<T>(sp->xv), in<T>(sp->dyv), out<T>(sp->dxv), gamma, mean, sink, pb.HW, set,
+                                status)));
+        else
+            BNS_BY_TYPE(pb.dtype,
+                        (launch(BNS_KERNEL_DIRECT_FIXUP, direct_finalize_fixup_kernel<T>, static_cast<unsigned>(pb.C),
+                                stream, in<T>(x), in<T>(dy), out<T>(dx), gamma, mean, sink, pb.HW, set, status)));
+        return last_error();
+    }
     launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
     // pass 2: the statistics terms, on S only
     const float inv_s = static_cast<float>(1.0 / pb.s);
@@ -654,10 +707,14 @@ int bns_set_tuning(const char* name, int value) {
         bool* bvalue;
     } knobs[] = {{"target_blocks", &g_target_blocks, nullptr},   {"min_chunk", &g_min_chunk, nullptr},
                  {"stat_target_blocks", &g_stat_target_blocks, nullptr}, {"stat_min_chunk", &g_stat_min_chunk, nullptr},
-                 {"pdl", nullptr, &g_pdl},                       {"l2_order", nullptr, &g_l2_order}};
+                 {"direct_max", &g_direct_max, nullptr},         {"pdl", nullptr, &g_pdl},                       {"l2_order", nullptr, &g_l2_order}};
     for (const Knob& k : knobs) {
         if (std::strcmp(name, k.name) != 0) continue;
         if (k.ivalue) {
+            if (k.ivalue == &g_direct_max && value == 0) {
+                g_direct_max = 0;
+                return BNS_OK;
+            }
             if (value < 1) return BNS_ERR_SHAPE;
             *k.ivalue = value;
         } else {
@@ -679,6 +736,8 @@ const char* bns_kernel_name(int kernel_kind) {
     case BNS_KERNEL_COL_FIXUP: return "col_fixup_kernel";
     case BNS_KERNEL_PATCH_FIXUP: return "patch_fixup_kernel";
     case BNS_KERNEL_MASK: return "selection_mask_kernel";
+    case BNS_KERNEL_DIRECT_MOMENTS: return "direct_moments_kernel";
+    case BNS_KERNEL_DIRECT_FIXUP: return "direct_finalize_fixup_kernel";
     }
     return "unknown";
 }

@@ -808,6 +808,116 @@ patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::
     }
 }
 
+// ------------------------------------------------------------------------------------ small sampled sets: one block per channel
+// When a channel's sampled set is small (a few thousand elements: small patches, a couple of virtual or
+// sampled samples) one block can read all of it, so the statistics need no partials and no finalize
+// launch, and in the backward the block that combines the channel's partial sums can apply the
+// statistics terms to the channel's sampled elements right away.  SampleSet enumerates the sampled
+// elements of a channel as q = 0 .. s-1.
+struct SampleSet {
+    int patches;       // 1: Feature Sampling patches of the real tensor; 0: whole rows (samples)
+    // whole rows: sample indices list[0..rows) or begin .. begin+rows-1; element q = (row q / HW, pixel q % HW)
+    const int* list;
+    int begin, rows;
+    // patches: element q = (sample q / (ph*pw), patch element q % (ph*pw))
+    PatchRule patch;
+    int N, C, H, W;
+    int s;             // elements per channel
+    __device__ __forceinline__ size_t at(int c, int q, unsigned* status) const {
+        const size_t HW = static_cast<size_t>(H) * W;
+        if (patches) {
+            const int PP = patch.ph * patch.pw;
+            const int n = q / PP, e = q - n * PP;
+            const int row = e / patch.pw, col = e - row * patch.pw;
+            int oh, ow;
+            patch_origin(patch, n, c, H, W, status, oh, ow);
+            return (static_cast<size_t>(n) * C + c) * HW + static_cast<size_t>(oh + row) * W + ow + col;
+        }
+        const int i = q / static_cast<int>(HW), hw = q - i * static_cast<int>(HW);
+        const int n = list ? list[i] : begin + i;
+        return (static_cast<size_t>(n) * C + c) * HW + hw;
+    }
+};
+
+// mean and invstd of channel blockIdx.x straight from its sampled elements.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+direct_moments_kernel(const typename T::storage* __restrict__ src, SampleSet set, float eps, float* __restrict__ mean,
+                      float* __restrict__ invstd, unsigned* status) {
+    __shared__ Moments s_warp[kThreads / 32];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x;
+    float K = 0.f, s1 = 0.f, s2 = 0.f, cnt = 0.f;
+    for (int q0 = threadIdx.x; q0 < set.s; q0 += kThreads * kUnroll) {
+        float v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int q = q0 + u * kThreads;
+            if (q < set.s) v[u] = to_float<T>(src[set.at(c, q, status)]);
+        }
+        if (cnt == 0.f) K = v[0];  // pivot: the thread's first value
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            if (q0 + u * kThreads < set.s) {
+                float d = v[u] - K;
+                s1 += d;
+                s2 = fmaf(d, d, s2);
+                cnt += 1.f;
+            }
+        }
+    }
+    Moments m = warp_merge(from_shifted_sums(cnt, K, s1, s2));
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        Moments acc = s_warp[0];
+        for (int w = 1; w < kThreads / 32; ++w) acc = merge(acc, s_warp[w]);
+        mean[c] = acc.mean;
+        invstd[c] = 1.0f / sqrtf(acc.m2 / static_cast<float>(set.s) + eps);
+    }
+}
+
+// Backward for a small sampled set: block c combines the partial sums of channel c (as the finalize
+// kernel would), publishes dgamma / dbeta, and rewrites the gradient of the channel's sampled elements
+// with the statistics terms: dst = a dy - A - Q (src - mean).  dy == NULL reads as zeros; dst == NULL
+// skips the rewrite.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+direct_finalize_fixup_kernel(const typename T::storage* __restrict__ src, const typename T::storage* __restrict__ dy,
+                             typename T::storage* __restrict__ dst, const float* __restrict__ gamma,
+                             const float* __restrict__ mean, GradSink G, int HW, SampleSet set, unsigned* status) {
+    __shared__ float s_grad[2];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x;
+    if (threadIdx.x < 32) warp_finish_grads(G, c, HW, threadIdx.x);  // lane 0 writes dgamma[c], dbeta[c]
+    __syncthreads();
+    if (!dst) return;
+    if (threadIdx.x == 0) {
+        s_grad[0] = G.dgamma[c];  // written by this thread just above
+        s_grad[1] = G.dbeta[c];
+    }
+    __syncthreads();
+    const FixCoef k = fix_coef(gamma[c], mean[c], G.invstd[c], s_grad[0], s_grad[1], 1.0f / static_cast<float>(set.s));
+    for (int q0 = threadIdx.x; q0 < set.s; q0 += kThreads * kUnroll) {
+        size_t at[kUnroll];
+        float g[kUnroll], xv[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int q = q0 + u * kThreads;
+            if (q < set.s) {
+                at[u] = set.at(c, q, status);
+                g[u] = dy ? to_float<T>(dy[at[u]]) : 0.f;
+                xv[u] = to_float<T>(src[at[u]]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (q0 + u * kThreads < set.s) dst[at[u]] = from_float<T>(fmaf(k.a, g[u], -k.A) - k.Q * (xv[u] - k.mu));
+    }
+}
+
 // ------------------------------------------------------------------------------------ selection mask (test aid)
 __global__ void __launch_bounds__(kThreads)
 selection_mask_kernel(uint8_t* __restrict__ mask, int rule, const int* __restrict__ list, int begin, int count,

@@ -216,3 +216,24 @@ def test_other_grid_shapes_still_match_the_oracle(target):
     finally:
         bns.set_tuning("target_blocks", 148 * 32)
         bns.set_tuning("stat_target_blocks", 148 * 8)
+
+
+@pytest.mark.parametrize("rule,kw", [
+    ("batch", dict(k=3, contiguous=False)), ("batch", dict(k=2)), ("feature", dict(ph=3, pw=3, offset_mode=0)),
+    ("feature", dict(ph=2, pw=4, offset_mode=2)), ("virtual", dict(nv=2)), ("virtual", dict(nv=1, with_dyv=False)),
+])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_small_sampled_sets_both_paths(rule, kw, dtype):
+    """A small sampled set is handled by one block per channel, a large one through partial sums and a
+    finalize launch; forcing either path on the same case must match the oracle."""
+    from paper_1810_10962_b200 import bns
+    kw = dict(kw)
+    if rule == "virtual":
+        kw["xv_dtype"] = dtype
+    case = make_case(24, 20, 14, 14, rule, seed=87, dtype=dtype, **kw)
+    try:
+        for direct_max in (0, 1 << 20):
+            bns.set_tuning("direct_max", direct_max)
+            compare(case, run_gpu(case))
+    finally:
+        bns.set_tuning("direct_max", 8192)
