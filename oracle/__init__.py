@@ -91,6 +91,10 @@ def _library():
         lib.oracle_forward.restype = None
         lib.oracle_backward.restype = None
         lib.oracle_selection_mask.restype = None
+        lib.oracle_forward_mixed.restype = None
+        lib.oracle_backward_mixed.restype = None
+        lib.oracle_moving_average.restype = None
+        lib.oracle_inference_forward.restype = None
         _lib = lib
     return _lib
 
@@ -212,3 +216,77 @@ def backward(x, dy, gamma, mean, var, eps, sp: Sampling, xv=None, dyv=None,
                                _ptr(var), ctypes.c_double(eps), ctypes.byref(c), _ptr(ch), nch, _ptr(dx),
                                _ptr(dxv), _ptr(dgamma), _ptr(dbeta))
     return Backward(dx, dxv, dgamma, dbeta)
+
+
+# ----------------------------------------------------------------------------- Eq. 4: VDN combined with a sampling rule
+@dataclass
+class ForwardMixed:
+    y: Optional[np.ndarray]
+    yv: Optional[np.ndarray]
+    mean: np.ndarray
+    var: np.ndarray
+    invstd: np.ndarray
+    mean_s: np.ndarray
+    var_s: np.ndarray
+    mean_v: np.ndarray
+    var_v: np.ndarray
+
+
+def forward_mixed(x, xv, gamma, beta, eps, mix, sp: Sampling, channels=None, want_y=True, want_yv=True) -> ForwardMixed:
+    """Eq. 4: E = mix*E[xv] + (1-mix)*E[x_s], Var likewise; Eq. 1 on x and xv with the mixed statistics."""
+    x, xv = _f32(x), _f32(xv)
+    N, C, H, W = x.shape
+    assert sp.rule in (RULE_BATCH, RULE_FEATURE) and xv.shape[1:] == (C, H, W)
+    _check_offsets(sp, N, C, H, W)
+    nv = xv.shape[0]
+    gamma, beta = _f32(gamma), _f32(beta)
+    ch, nch = _channels(channels, C)
+    y = np.empty((N, nch, H, W), dtype=np.float64) if want_y else None
+    yv = np.empty((nv, nch, H, W), dtype=np.float64) if want_yv else None
+    vec = [np.empty(nch, dtype=np.float64) for _ in range(6)]
+    c, _keep = sp._c()
+    _library().oracle_forward_mixed(N, C, H, W, _ptr(x), _ptr(xv), nv, _ptr(gamma), _ptr(beta), ctypes.c_double(eps),
+                                    ctypes.c_double(mix), ctypes.byref(c), _ptr(ch), nch, _ptr(y), _ptr(yv),
+                                    *[_ptr(v) for v in vec])
+    mean, var, mean_s, var_s, mean_v, var_v = vec
+    return ForwardMixed(y, yv, mean, var, 1.0 / np.sqrt(var + eps), mean_s, var_s, mean_v, var_v)
+
+
+def backward_mixed(x, xv, dy, dyv, gamma, fwd: ForwardMixed, eps, mix, sp: Sampling, channels=None) -> Backward:
+    """Chain rule through Eq. 4 (see bns_oracle.c); `fwd` is forward_mixed's result for the same channels."""
+    x, xv, dy, dyv = _f32(x), _f32(xv), _f32(dy), _f32(dyv)
+    N, C, H, W = x.shape
+    nv = xv.shape[0]
+    gamma = _f32(gamma)
+    ch, nch = _channels(channels, C)
+    dx = np.empty((N, nch, H, W), dtype=np.float64)
+    dxv = np.empty((nv, nch, H, W), dtype=np.float64)
+    dgamma, dbeta = (np.empty(nch, dtype=np.float64) for _ in range(2))
+    c, _keep = sp._c()
+    _library().oracle_backward_mixed(N, C, H, W, _ptr(x), _ptr(xv), nv, _ptr(dy), _ptr(dyv), _ptr(gamma),
+                                     _ptr(fwd.mean), _ptr(fwd.var), _ptr(fwd.mean_s), _ptr(fwd.mean_v),
+                                     ctypes.c_double(eps), ctypes.c_double(mix), ctypes.byref(c), _ptr(ch), nch,
+                                     _ptr(dx), _ptr(dxv), _ptr(dgamma), _ptr(dbeta))
+    return Backward(dx, dxv, dgamma, dbeta)
+
+
+# ----------------------------------------------------------------------------- Appendix D: moving average, validation forward
+def moving_average(X, X_ma, alpha, first_iteration) -> np.ndarray:
+    """Eq. 8: returns the updated moving average (X_ma is not modified)."""
+    X = np.ascontiguousarray(X, dtype=np.float64)
+    out = np.array(X_ma, dtype=np.float64, copy=True) if X_ma is not None else np.zeros_like(X)
+    _library().oracle_moving_average(X.size, int(bool(first_iteration)), ctypes.c_double(alpha), _ptr(X), _ptr(out))
+    return out
+
+
+def inference_forward(x, gamma, beta, eps, E_ma, Var_ma) -> np.ndarray:
+    """Eq. 1 with the recorded moving averages in place of the batch statistics."""
+    x = _f32(x)
+    N, C, H, W = x.shape
+    gamma, beta = _f32(gamma), _f32(beta)
+    E_ma = np.ascontiguousarray(E_ma, dtype=np.float64)
+    Var_ma = np.ascontiguousarray(Var_ma, dtype=np.float64)
+    y = np.empty(x.shape, dtype=np.float64)
+    _library().oracle_inference_forward(N, C, H, W, _ptr(x), _ptr(gamma), _ptr(beta), ctypes.c_double(eps), _ptr(E_ma),
+                                        _ptr(Var_ma), _ptr(y))
+    return y

@@ -15,6 +15,8 @@
  *   Algorithm 1  NS/BS slice  B[begin : begin+n_s-1, :, :, :]   (here: an explicit sample list)
  *   Algorithm 2  FS slice     B[:, bh : bh+h_s-1, bw : bw+w_s-1, :]
  *   Algorithm 3  VDN          statistics from the virtual rows only
+ *   Eq. 4  VDN combined with a sampling rule   X = b X[x_v] + (1-b) X[x_s],  X in {E, Var}
+ *   Eq. 8  moving average of E and Var for validation (Appendix D)
  * Layout is NCHW (the paper writes NHWC; the reduction is over N, H, W for each channel).
  *
  * Inputs are float arrays (bf16 data is widened exactly by the caller); all arithmetic is double.
@@ -251,4 +253,168 @@ double oracle_adder_tree_depth_ratio(int N, int H, int W, const oracle_sampling 
     double m = (double)N * H * W;
     double s = (double)oracle_sample_count(N, H, W, sp);
     return log(m) / log(s);
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Eq. 4: statistics mixed from the virtual samples and a sampling rule of the real batch,
+ *   E = b E[x_v] + (1-b) E[x_s],   Var = b Var[x_v] + (1-b) Var[x_s]
+ * where each variance is taken about its own mean (Eq. 3 applied to each set).  sp is the rule of
+ * the real batch (BATCH or FEATURE); the virtual set is all of xv [nv,C,H,W].  Every real and every
+ * virtual element is normalised with the mixed statistics (Eq. 1).
+ * Outputs, compact over the requested channels: y [N,nch,H,W], yv [nv,nch,H,W] (may be NULL),
+ * mean/var (mixed), mean_s/var_s (sampled real set), mean_v/var_v (virtual set), each [nch].
+ */
+void oracle_forward_mixed(int N, int C, int H, int W, const float *x, const float *xv, int nv,
+                          const float *gamma, const float *beta, double eps, double b,
+                          const oracle_sampling *sp, const int32_t *channels, int nch,
+                          double *y, double *yv, double *mean, double *var,
+                          double *mean_s, double *var_s, double *mean_v, double *var_v)
+{
+    if (!channels) nch = C;
+    const double s_s = (double)oracle_sample_count(N, H, W, sp);
+    const double s_v = (double)nv * H * W;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int j = 0; j < nch; ++j) {
+        const int c = channels ? channels[j] : j;
+        /* Eq. 3 on the sampled real set */
+        double sum = 0.0, sq = 0.0;
+        for (int n = 0; n < N; ++n)
+            for (int h = 0; h < H; ++h)
+                for (int w = 0; w < W; ++w)
+                    if (in_S(sp, C, n, c, h, w)) sum += (double)x[AT(n, c, h, w)];
+        const double E_s = sum / s_s;
+        for (int n = 0; n < N; ++n)
+            for (int h = 0; h < H; ++h)
+                for (int w = 0; w < W; ++w)
+                    if (in_S(sp, C, n, c, h, w)) {
+                        double d = (double)x[AT(n, c, h, w)] - E_s;
+                        sq += d * d;
+                    }
+        const double Var_s = sq / s_s;
+        /* Eq. 3 on the virtual set */
+        sum = 0.0, sq = 0.0;
+        for (int n = 0; n < nv; ++n)
+            for (int h = 0; h < H; ++h)
+                for (int w = 0; w < W; ++w) sum += (double)xv[AT(n, c, h, w)];
+        const double E_v = sum / s_v;
+        for (int n = 0; n < nv; ++n)
+            for (int h = 0; h < H; ++h)
+                for (int w = 0; w < W; ++w) {
+                    double d = (double)xv[AT(n, c, h, w)] - E_v;
+                    sq += d * d;
+                }
+        const double Var_v = sq / s_v;
+        /* Eq. 4 */
+        const double E = b * E_v + (1.0 - b) * E_s;
+        const double Var = b * Var_v + (1.0 - b) * Var_s;
+        mean[j] = E, var[j] = Var;
+        mean_s[j] = E_s, var_s[j] = Var_s;
+        mean_v[j] = E_v, var_v[j] = Var_v;
+        /* Eq. 1 */
+        const double g = (double)gamma[c], bt = (double)beta[c];
+        if (y)
+            for (int n = 0; n < N; ++n)
+                for (int h = 0; h < H; ++h)
+                    for (int w = 0; w < W; ++w)
+                        y[OUT(n, j, h, w)] = g * (((double)x[AT(n, c, h, w)] - E) / sqrt(Var + eps)) + bt;
+        if (yv)
+            for (int n = 0; n < nv; ++n)
+                for (int h = 0; h < H; ++h)
+                    for (int w = 0; w < W; ++w)
+                        yv[OUT(n, j, h, w)] = g * (((double)xv[AT(n, c, h, w)] - E) / sqrt(Var + eps)) + bt;
+    }
+}
+
+/*
+ * Backward of the mixed statistics, by the chain rule through Eq. 4 in the notation of Eq. 5/6.
+ * dl/dE and dl/dVar are the full-length sums of Eq. 5 over every normalised element (the real batch
+ * and, when dyv is given, the virtual rows).  Var does not depend on E here (each variance is about
+ * its own mean), and d Var_s / d E_s = -(2/s_s) sum_S (x - E_s) = 0, so
+ *   dl/dE_s = (1-b) dl/dE,  dl/dVar_s = (1-b) dl/dVar,  dl/dE_v = b dl/dE,  dl/dVar_v = b dl/dVar,
+ *   dx_i  = dl/dx^_i / sqrt(Var+eps) + [i in S] ( dl/dE_s / s_s + dl/dVar_s 2 (x_i - E_s) / s_s )
+ *   dxv_i = dl/dx^v_i / sqrt(Var+eps) +           dl/dE_v / s_v + dl/dVar_v 2 (xv_i - E_v) / s_v
+ */
+void oracle_backward_mixed(int N, int C, int H, int W, const float *x, const float *xv, int nv,
+                           const float *dy, const float *dyv, const float *gamma,
+                           const double *mean, const double *var, const double *mean_s, const double *mean_v,
+                           double eps, double b, const oracle_sampling *sp,
+                           const int32_t *channels, int nch,
+                           double *dx, double *dxv, double *dgamma, double *dbeta)
+{
+    if (!channels) nch = C;
+    const double s_s = (double)oracle_sample_count(N, H, W, sp);
+    const double s_v = (double)nv * H * W;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int j = 0; j < nch; ++j) {
+        const int c = channels ? channels[j] : j;
+        const double E = mean[j], Var = var[j], E_s = mean_s[j], E_v = mean_v[j], g = (double)gamma[c];
+        double dl_dE = 0.0, dl_dVar = 0.0, dl_dgamma = 0.0, dl_dbeta = 0.0;
+        for (int n = 0; n < N; ++n)
+            for (int h = 0; h < H; ++h)
+                for (int w = 0; w < W; ++w) {
+                    double dyi = (double)dy[AT(n, c, h, w)], xi = (double)x[AT(n, c, h, w)];
+                    double dl_dxhat = dyi * g;
+                    dl_dE += dl_dxhat * (-1.0 / sqrt(Var + eps));
+                    dl_dVar += dl_dxhat * (xi - E) * (-0.5) * pow(Var + eps, -1.5);
+                    dl_dgamma += dyi * ((xi - E) / sqrt(Var + eps));
+                    dl_dbeta += dyi;
+                }
+        if (dyv)
+            for (int n = 0; n < nv; ++n)
+                for (int h = 0; h < H; ++h)
+                    for (int w = 0; w < W; ++w) {
+                        double dyi = (double)dyv[AT(n, c, h, w)], xi = (double)xv[AT(n, c, h, w)];
+                        double dl_dxhat = dyi * g;
+                        dl_dE += dl_dxhat * (-1.0 / sqrt(Var + eps));
+                        dl_dVar += dl_dxhat * (xi - E) * (-0.5) * pow(Var + eps, -1.5);
+                        dl_dgamma += dyi * ((xi - E) / sqrt(Var + eps));
+                        dl_dbeta += dyi;
+                    }
+        dgamma[j] = dl_dgamma;
+        dbeta[j] = dl_dbeta;
+        const double dl_dE_s = (1.0 - b) * dl_dE, dl_dVar_s = (1.0 - b) * dl_dVar;
+        const double dl_dE_v = b * dl_dE, dl_dVar_v = b * dl_dVar;
+        if (dx)
+            for (int n = 0; n < N; ++n)
+                for (int h = 0; h < H; ++h)
+                    for (int w = 0; w < W; ++w) {
+                        double dyi = (double)dy[AT(n, c, h, w)], xi = (double)x[AT(n, c, h, w)];
+                        double v = dyi * g / sqrt(Var + eps);
+                        if (in_S(sp, C, n, c, h, w)) v += dl_dE_s / s_s + dl_dVar_s * 2.0 * (xi - E_s) / s_s;
+                        dx[OUT(n, j, h, w)] = v;
+                    }
+        if (dxv)
+            for (int n = 0; n < nv; ++n)
+                for (int h = 0; h < H; ++h)
+                    for (int w = 0; w < W; ++w) {
+                        double dyi = dyv ? (double)dyv[AT(n, c, h, w)] : 0.0;
+                        double xi = (double)xv[AT(n, c, h, w)];
+                        dxv[OUT(n, j, h, w)] = dyi * g / sqrt(Var + eps) + dl_dE_v / s_v +
+                                               dl_dVar_v * 2.0 * (xi - E_v) / s_v;
+                    }
+    }
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Appendix D, Eq. 8: the recorded moving average of a statistic X (E or Var) over iterations:
+ * X_ma = X at the first iteration, alpha X + (1 - alpha) X_ma afterwards (alpha weights the NEW value).
+ */
+void oracle_moving_average(int C, int first_iteration, double alpha, const double *X, double *X_ma)
+{
+    for (int c = 0; c < C; ++c) X_ma[c] = first_iteration ? X[c] : alpha * X[c] + (1.0 - alpha) * X_ma[c];
+}
+
+/* Validation step (Appendix D): Eq. 1 with E and Var replaced by the recorded moving averages. */
+void oracle_inference_forward(int N, int C, int H, int W, const float *x, const float *gamma,
+                              const float *beta, double eps, const double *E_ma, const double *Var_ma,
+                              double *y)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int c = 0; c < C; ++c)
+        for (int n = 0; n < N; ++n)
+            for (int h = 0; h < H; ++h)
+                for (int w = 0; w < W; ++w) {
+                    double xhat = ((double)x[AT(n, c, h, w)] - E_ma[c]) / sqrt(Var_ma[c] + eps);
+                    y[AT(n, c, h, w)] = (double)gamma[c] * xhat + (double)beta[c];
+                }
 }

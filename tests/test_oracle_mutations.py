@@ -30,6 +30,14 @@ MUTANTS = [
     ("xhat_without_centering", "dl_dgamma += dyi * ((xi - E) * istd);\n                    dl_dbeta += dyi;\n                }\n        if (virt",
      "dl_dgamma += dyi * (xi * istd);\n                    dl_dbeta += dyi;\n                }\n        if (virt"),
     ("virtual_rows_not_in_sums", "if (virt && dyv)", "if (0 && dyv)"),
+    # Eq. 4 and Appendix D
+    ("mixed_weights_swapped", "const double E = b * E_v + (1.0 - b) * E_s;", "const double E = b * E_s + (1.0 - b) * E_v;"),
+    ("mixed_correction_about_mixed_mean", "v += dl_dE_s / s_s + dl_dVar_s * 2.0 * (xi - E_s) / s_s;",
+     "v += dl_dE_s / s_s + dl_dVar_s * 2.0 * (xi - E) / s_s;"),
+    ("mixed_virtual_share_dropped", "const double dl_dE_v = b * dl_dE, dl_dVar_v = b * dl_dVar;",
+     "const double dl_dE_v = dl_dE, dl_dVar_v = dl_dVar;"),
+    ("moving_average_alpha_on_old_value", "alpha * X[c] + (1.0 - alpha) * X_ma[c]", "(1.0 - alpha) * X[c] + alpha * X_ma[c]"),
+    ("inference_eps_outside_root", "/ sqrt(Var_ma[c] + eps);", "/ (sqrt(Var_ma[c]) + eps);"),
 ]
 
 
@@ -43,7 +51,8 @@ def test_planted_mistake_is_caught(tmp_path, name, old, new):
     compile_source(str(src), str(lib))
     env = dict(os.environ, BNS_ORACLE_LIBRARY=str(lib))
     run = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
-                          os.path.join(ROOT, "tests", "test_oracle_pins.py")],
+                          os.path.join(ROOT, "tests", "test_oracle_pins.py"),
+                          os.path.join(ROOT, "tests", "test_oracle_next_rows.py")],
                          cwd=ROOT, env=env, capture_output=True, text=True)
     assert run.returncode != 0, f"no pin noticed the planted mistake '{name}'"
     assert "failed" in run.stdout
