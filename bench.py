@@ -65,7 +65,7 @@ class Layer:
             return m
         if self.rule == "batch":
             return self.kw["k"] * self.H * self.W
-        if self.rule == "feature":
+        if self.rule in ("feature", "mixed"):
             return self.N * self.kw["ph"] * self.kw["pw"]
         return self.kw["nv"] * self.H * self.W
 
@@ -75,6 +75,10 @@ class Layer:
         vec = 16 * C
         if self.rule == "full":
             return 8 * E * b + 2 * vec
+        if self.rule == "mixed":
+            ev = self.kw["nv"] * C * self.H * self.W * 4      # xv is fp32: statistics, yv, and dxv as for VDN
+            r = self.sampled_per_channel() / (self.N * self.H * self.W)
+            return int(round((5 + 4 * r) * E * b)) + 5 * ev + 2 * vec
         if self.rule == "virtual":
             ev = self.kw["nv"] * C * self.H * self.W * 4      # xv is fp32
             # forward: read xv (statistics), read xv + write yv, read x, write y; backward: read x, dy, write dx,
@@ -100,6 +104,9 @@ def workload_layers(name):
             p = max(1, H // 8)
             layers.append(Layer(f"fs{p}x{p}_c{C}_h{H}", 256, C, H, H, "bf16", "feature", count=cnt, ph=p, pw=p))
         return layers
+    if name == "fs_vdn":
+        # the paper's most accurate variant (Table 2, "FS+VDN"): Eq. 4 with a patch and two virtual samples
+        return [Layer("fs8x8_vdn2", 256, 64, 56, 56, "f32", "mixed", ph=8, pw=8, nv=2, mix=0.5)]
     if name == "tiny":
         return [Layer("bs2", 8, 16, 8, 8, "f32", "batch", k=2)]
     raise SystemExit(f"unknown workload {name}")
@@ -118,7 +125,7 @@ def selected_layers(args):
 
 
 def layer_seed(workload, index):
-    return 1810 + 100 * (["tiny", "cifar", "resnet18_stage1", "vdn", "resnet50"].index(workload) + 1) + index
+    return 1810 + 100 * (["tiny", "cifar", "resnet18_stage1", "vdn", "resnet50", "fs_vdn"].index(workload) + 1) + index
 
 
 def host_inputs(layer: Layer, seed):
@@ -136,6 +143,9 @@ def host_inputs(layer: Layer, seed):
     elif layer.rule == "feature":
         extra["offsets"] = I.patch_offsets(N, C, H, W, layer.kw["ph"], layer.kw["pw"], I.OFFSETS_SHARED, seed)
     elif layer.rule == "virtual":
+        extra["xv"] = I.virtual_samples(layer.kw["nv"], C, H, W, seed)
+    elif layer.rule == "mixed":
+        extra["offsets"] = I.patch_offsets(N, C, H, W, layer.kw["ph"], layer.kw["pw"], I.OFFSETS_SHARED, seed)
         extra["xv"] = I.virtual_samples(layer.kw["nv"], C, H, W, seed)
     return dict(x=x, dy=dy, gamma=gamma, beta=beta, **extra)
 
@@ -208,6 +218,7 @@ class DeviceLayer:
     def __init__(self, layer: Layer, host, sets, torch, bns, full_bn=False):
         self.layer, self.bns, self.torch = layer, bns, torch
         self.full = full_bn or layer.rule == "full"
+        self.mixed = layer.rule == "mixed" and not self.full
         dt = torch.float32 if layer.dtype == "f32" else torch.bfloat16
 
         def dev(a):
@@ -226,6 +237,13 @@ class DeviceLayer:
             self.sp = bns.Sampling.batch(host["sample_idx"])
         elif layer.rule == "feature":
             self.sp = bns.Sampling.feature(layer.kw["ph"], layer.kw["pw"], host["offsets"])
+        elif layer.rule == "mixed":
+            xv = torch.from_numpy(host["xv"]).cuda()
+            self.sp = bns.Sampling.feature(layer.kw["ph"], layer.kw["pw"], host["offsets"]).with_virtual(
+                xv, yv=torch.empty_like(xv), dyv=None, dxv=torch.empty_like(xv))
+            self.mean_s, self.mean_v = (torch.empty(C, device="cuda") for _ in range(2))
+            self.ws = torch.empty(bns.workspace_bytes_mixed(x, self.sp), dtype=torch.uint8, device="cuda")
+            return
         else:
             xv = torch.from_numpy(host["xv"]).cuda()
             self.sp = bns.Sampling.virtual(xv, yv=torch.empty_like(xv), dyv=None, dxv=torch.empty_like(xv))
@@ -236,6 +254,14 @@ class DeviceLayer:
                       for sx, sdy, sy, sdx in self.sets]
 
     def step(self, i):
+        if self.mixed:
+            x, dy, y, dx = self.sets[i % len(self.sets)]
+            b, mix = self.bns, self.layer.kw["mix"]
+            b.forward_mixed(x, self.gamma, self.beta, EPS, mix, self.sp, workspace=self.ws, y=y,
+                            stats=(self.mean, self.invstd, self.mean_s, self.mean_v))
+            b.backward_mixed(x, dy, self.gamma, self.mean, self.invstd, self.mean_s, self.mean_v, mix, self.sp,
+                             workspace=self.ws, dx=dx, grads=(self.dgamma, self.dbeta))
+            return
         call = self.calls[i % len(self.calls)]
         call.forward()
         call.backward()
@@ -468,7 +494,7 @@ def run_e2e(torch, bns, layers, hosts, steps):
     """Same metric through bns_forward_backward_host: pinned host tensors in, pinned host tensors out."""
     items, h2d, d2h = [], 0, 0
     for l, h in zip(layers, hosts):
-        if l.rule == "virtual":
+        if l.rule in ("virtual", "mixed"):
             return None      # the host entry point keeps xv on the device; not measured end to end
         dt = torch.float32 if l.dtype == "f32" else torch.bfloat16
         pin = lambda a: torch.from_numpy(a).to(dt).pin_memory()
@@ -525,6 +551,12 @@ def oracle_sample(layers, hosts, seconds):
         else:
             sp = O.Sampling.full()
         ch = np.asarray(channels, dtype=np.int32)
+        if l.rule == "mixed":
+            sp = O.Sampling.feature(l.kw["ph"], l.kw["pw"], h["offsets"])
+            t0 = time.perf_counter()
+            f = O.forward_mixed(h["x"], h["xv"], h["gamma"], h["beta"], EPS, l.kw["mix"], sp, channels=ch)
+            O.backward_mixed(h["x"], h["xv"], h["dy"], None, h["gamma"], f, EPS, l.kw["mix"], sp, channels=ch)
+            return time.perf_counter() - t0
         t0 = time.perf_counter()
         f = O.forward(h["x"], h["gamma"], h["beta"], EPS, sp, xv=h.get("xv"), channels=ch)
         O.backward(h["x"], h["dy"], h["gamma"], f.mean, f.var, EPS, sp, xv=h.get("xv"), channels=ch)
@@ -595,7 +627,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="resnet18_stage1",
-                    choices=["resnet18_stage1", "cifar", "vdn", "resnet50", "tiny"])
+                    choices=["resnet18_stage1", "cifar", "vdn", "resnet50", "fs_vdn", "tiny"])
     ap.add_argument("--only", default=None, help="comma-separated layer names: run just these layers of the workload")
     ap.add_argument("--tune", action="append", default=[], metavar="NAME=VALUE",
                     help="launch-shape knob of the library (bns_set_tuning), e.g. --tune pdl=0")

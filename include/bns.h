@@ -130,6 +130,48 @@ bns_status bns_full_bn(const bns_shape* shape, const void* x, const float* gamma
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Virtual Dataset Normalization combined with a sampling rule (Eq. 4 of the paper, its most accurate
+ * variant, "FS+VDN"):   X = mix X[x_v] + (1 - mix) X[x_s]   for X in {E, Var},
+ * where x_s is the sampled set of the real batch (`sampling->rule` BATCH or FEATURE) and x_v the nv
+ * virtual samples `sampling->xv` (the VIRTUAL fields of bns_sampling are used as well); each variance
+ * is taken about its own mean (Eq. 3 on each set).  The paper uses mix = 0.5.  x and, if yv is given,
+ * xv are normalised with the mixed statistics (Eq. 1).
+ * Forward writes y, mean[C] and invstd[C] (mixed) and the two means mean_s[C], mean_v[C], which the
+ * backward needs.  The paper derives no gradient for Eq. 4; by the chain rule through it,
+ *   dx_i  = gamma invstd dy_i   - [i in S] (1-mix) gamma invstd (dbeta + invstd (x_i - mean_s) dgamma) / s_s
+ *   dxv_i = gamma invstd dyv_i  -             mix  gamma invstd (dbeta + invstd (xv_i - mean_v) dgamma) / s_v
+ * with dbeta, dgamma the full-length sums of Eq. 5 over the real batch and (if dyv is given) the
+ * virtual rows.  Workspace: bns_workspace_bytes_mixed().  mix must lie in [0,1].
+ */
+size_t bns_workspace_bytes_mixed(const bns_shape* shape, const bns_sampling* sampling);
+bns_status bns_forward_mixed(const bns_shape* shape, const void* x, const float* gamma, const float* beta,
+                             float eps, float mix, const bns_sampling* sampling, void* y, float* mean,
+                             float* invstd, float* mean_s, float* mean_v,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+bns_status bns_backward_mixed(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
+                              const float* mean, const float* invstd, const float* mean_s, const float* mean_v,
+                              float mix, const bns_sampling* sampling, void* dx, float* dgamma, float* dbeta,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Moving average of the statistics for validation (Appendix D, Eq. 8):
+ *   X_ma = X at the first iteration,  alpha X + (1 - alpha) X_ma afterwards,  X in {E, Var}
+ * (alpha weights the NEW value, as Eq. 8 and Eq. 9 state it; the paper finds 0.7 best for
+ * BS-1/128).  mean and invstd are a forward call's outputs; Var is recovered as 1/invstd^2 - eps.
+ * mean_ma[C], var_ma[C] are updated in place (read only when first_iteration == 0).
+ */
+bns_status bns_update_moving_average(int C, const float* mean, const float* invstd, float eps, float alpha,
+                                     int first_iteration, float* mean_ma, float* var_ma, void* cuda_stream);
+
+/*
+ * Validation-time forward (Appendix D): Eq. 1 with E and Var replaced by the recorded moving
+ * averages, y = gamma (x - mean_ma) / sqrt(var_ma + eps) + beta.  Workspace as for bns_full_bn.
+ */
+bns_status bns_inference_forward(const bns_shape* shape, const void* x, const float* gamma, const float* beta,
+                                 float eps, const float* mean_ma, const float* var_ma, void* y,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * bns_forward for callers that cannot provide scratch memory.  (The paper has no counterpart; this
  * is a packaging variant of bns_forward: same kernels, same results.)
  *
@@ -200,7 +242,8 @@ typedef enum {
     BNS_KERNEL_MASK = 8,
     BNS_KERNEL_DIRECT_MOMENTS = 9, /* statistics of a small sampled set, one block per channel    */
     BNS_KERNEL_DIRECT_FIXUP = 10,  /* backward sums combined + statistics terms, small sampled set */
-    BNS_KERNEL_KINDS = 11
+    BNS_KERNEL_VECTOR = 11,        /* C-length kernels: mixing of statistics, moving average          */
+    BNS_KERNEL_KINDS = 12
 } bns_kernel_kind;
 
 /* Number of kernels this library has launched in this process since load (or since reset). */

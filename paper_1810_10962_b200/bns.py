@@ -23,16 +23,18 @@ RULE_FULL, RULE_BATCH, RULE_FEATURE, RULE_VIRTUAL = 0, 1, 2, 3
 OFF_SHARED, OFF_PER_SAMPLE, OFF_PER_MAP = 0, 1, 2
 FLAG_BAD_OFFSET = 1
 
-KERNEL_KINDS = 11
+KERNEL_KINDS = 12
 (KERNEL_COL_MOMENTS, KERNEL_PATCH_MOMENTS, KERNEL_FINALIZE_STATS, KERNEL_NORMALIZE, KERNEL_BWD_REDUCE,
  KERNEL_FINALIZE_BWD, KERNEL_COL_FIXUP, KERNEL_PATCH_FIXUP, KERNEL_MASK, KERNEL_DIRECT_MOMENTS,
- KERNEL_DIRECT_FIXUP) = range(KERNEL_KINDS)
+ KERNEL_DIRECT_FIXUP, KERNEL_VECTOR) = range(KERNEL_KINDS)
 
 EXPORTS = [
     "bns_workspace_bytes", "bns_forward", "bns_forward_static", "bns_static_workspace_bytes", "bns_backward", "bns_full_bn", "bns_host_arena_bytes",
     "bns_forward_backward_host", "bns_debug_selection_mask", "bns_workspace_status", "bns_status_string",
     "bns_launch_count", "bns_launch_count_reset", "bns_profile_enable", "bns_profile_read", "bns_kernel_name",
     "bns_set_tuning",
+    "bns_workspace_bytes_mixed", "bns_forward_mixed", "bns_backward_mixed", "bns_update_moving_average",
+    "bns_inference_forward",
 ]
 
 
@@ -107,6 +109,16 @@ def load():
     lib.bns_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float)]
     lib.bns_kernel_name.restype = ctypes.c_char_p
     lib.bns_kernel_name.argtypes = [ctypes.c_int]
+    lib.bns_workspace_bytes_mixed.restype = sz
+    lib.bns_workspace_bytes_mixed.argtypes = [shp, smp]
+    lib.bns_forward_mixed.restype = ctypes.c_int
+    lib.bns_forward_mixed.argtypes = [shp, vp, vp, vp, fl, fl, smp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.bns_backward_mixed.restype = ctypes.c_int
+    lib.bns_backward_mixed.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, fl, smp, vp, vp, vp, vp, sz, vp]
+    lib.bns_update_moving_average.restype = ctypes.c_int
+    lib.bns_update_moving_average.argtypes = [ctypes.c_int, vp, vp, fl, fl, ctypes.c_int, vp, vp, vp]
+    lib.bns_inference_forward.restype = ctypes.c_int
+    lib.bns_inference_forward.argtypes = [shp, vp, vp, vp, fl, vp, vp, vp, vp, sz, vp]
     lib.bns_set_tuning.restype = ctypes.c_int
     lib.bns_set_tuning.argtypes = [ctypes.c_char_p, ctypes.c_int]
     _lib = lib
@@ -153,6 +165,11 @@ class Sampling:
     def virtual(xv, yv=None, dyv=None, dxv=None):
         return Sampling(RULE_VIRTUAL, nv=int(xv.shape[0]), xv=xv, yv=yv, dyv=dyv, dxv=dxv)
 
+    def with_virtual(self, xv, yv=None, dyv=None, dxv=None):
+        """This BATCH / FEATURE rule combined with virtual samples (for forward_mixed / backward_mixed)."""
+        return Sampling(self.rule, sample_idx=self.sample_idx, ph=self.ph, pw=self.pw, offset_mode=self.offset_mode,
+                        offsets=self.offsets, nv=int(xv.shape[0]), xv=xv, yv=yv, dyv=dyv, dxv=dxv)
+
     def _c(self) -> _Sampling:
         c = _Sampling()
         c.rule = self.rule
@@ -168,8 +185,8 @@ class Sampling:
                 if not (isinstance(off, torch.Tensor) and off.is_cuda and off.dtype == torch.int32 and off.is_contiguous()):
                     raise TypeError("per-sample / per-map offsets must be a contiguous CUDA int32 tensor")
                 c.offsets = off.data_ptr()
-        elif self.rule == RULE_VIRTUAL:
-            c.nv = self.nv
+        if self.xv is not None:      # the VIRTUAL rule, or a sampling rule combined with virtual samples (Eq. 4)
+            c.nv = int(self.xv.shape[0])
             c.xv_dtype = _dtype_code(self.xv)
             c.xv = _dev(self.xv)
             for name in ("yv", "dyv", "dxv"):
@@ -358,6 +375,69 @@ class Prepared:
                                     torch.cuda.current_stream().cuda_stream)
         if st != OK:
             raise BnsError(st, "bns_backward")
+
+
+# ----------------------------------------------------------------------------- Eq. 4 and Appendix D
+def workspace_bytes_mixed(x, sampling: Sampling) -> int:
+    sh, sp = _shape(x), sampling._c()
+    n = load().bns_workspace_bytes_mixed(ctypes.byref(sh), ctypes.byref(sp))
+    if n == 0:
+        raise BnsError(-3, "bns_workspace_bytes_mixed (invalid shape or sampling rule)")
+    return int(n)
+
+
+def forward_mixed(x, gamma, beta, eps, mix, sampling: Sampling, workspace=None, y=None, stats=None):
+    """bns_forward_mixed: returns (y, mean, invstd, mean_s, mean_v); yv goes to sampling.yv.  `stats` may
+    give the four float32[C] output tensors (mean, invstd, mean_s, mean_v)."""
+    sh, sp = _shape(x), sampling._c()
+    C = x.shape[1]
+    y = torch.empty_like(x) if y is None else y
+    mean, invstd, mean_s, mean_v = stats if stats is not None else (
+        torch.empty(C, dtype=torch.float32, device=x.device) for _ in range(4))
+    if workspace is None:
+        workspace = torch.empty(workspace_bytes_mixed(x, sampling), dtype=torch.uint8, device=x.device)
+    st = load().bns_forward_mixed(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), float(mix),
+                                  ctypes.byref(sp), _dev(y), _vec(mean, C), _vec(invstd, C), _vec(mean_s, C),
+                                  _vec(mean_v, C), workspace.data_ptr(), workspace.numel(), _stream())
+    _check(st, "bns_forward_mixed")
+    return y, mean, invstd, mean_s, mean_v
+
+
+def backward_mixed(x, dy, gamma, mean, invstd, mean_s, mean_v, mix, sampling: Sampling, workspace=None, dx=None,
+                   grads=None):
+    """bns_backward_mixed: returns (dx, dgamma, dbeta); dxv goes to sampling.dxv."""
+    sh, sp = _shape(x), sampling._c()
+    C = x.shape[1]
+    dx = torch.empty_like(x) if dx is None else dx
+    dgamma, dbeta = grads if grads is not None else (
+        torch.empty(C, dtype=torch.float32, device=x.device) for _ in range(2))
+    if workspace is None:
+        workspace = torch.empty(workspace_bytes_mixed(x, sampling), dtype=torch.uint8, device=x.device)
+    st = load().bns_backward_mixed(ctypes.byref(sh), _dev(x), _dev(dy), _vec(gamma, C), _vec(mean, C), _vec(invstd, C),
+                                   _vec(mean_s, C), _vec(mean_v, C), float(mix), ctypes.byref(sp), _dev(dx),
+                                   _vec(dgamma, C), _vec(dbeta, C), workspace.data_ptr(), workspace.numel(), _stream())
+    _check(st, "bns_backward_mixed")
+    return dx, dgamma, dbeta
+
+
+def update_moving_average(mean, invstd, eps, alpha, first_iteration, mean_ma, var_ma):
+    """bns_update_moving_average: Eq. 8 on mean_ma / var_ma, in place."""
+    C = mean.numel()
+    st = load().bns_update_moving_average(C, _vec(mean, C), _vec(invstd, C), float(eps), float(alpha),
+                                          1 if first_iteration else 0, _vec(mean_ma, C), _vec(var_ma, C), _stream())
+    _check(st, "bns_update_moving_average")
+
+
+def inference_forward(x, gamma, beta, eps, mean_ma, var_ma, y=None, workspace=None):
+    """bns_inference_forward: Eq. 1 with the recorded moving averages; returns y."""
+    sh = _shape(x)
+    C = x.shape[1]
+    y = torch.empty_like(x) if y is None else y
+    ws, wp, wn = _workspace(x, Sampling.full(), workspace)
+    st = load().bns_inference_forward(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps),
+                                      _vec(mean_ma, C), _vec(var_ma, C), _dev(y), wp, wn, _stream())
+    _check(st, "bns_inference_forward")
+    return y
 
 
 # ----------------------------------------------------------------------------- host-buffer step

@@ -520,6 +520,118 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
     return last_error();
 }
 
+// ------------------------------------------------------------------------------------ Eq. 4: VDN combined with a sampling rule
+// Two problems over the same shape: the sampling rule of the real batch (BATCH or FEATURE) and the
+// virtual samples.  Workspace: [rule's workspace | virtual workspace | 2 C floats].
+struct MixedProblem {
+    Problem real, virt;
+    bns_sampling virt_rule;
+    size_t off_virt, off_vec, total;
+};
+
+bns_status make_mixed(const bns_shape* sh, const bns_sampling* sp, float mix, MixedProblem& mp) {
+    if (!sp) return BNS_ERR_NULL;
+    if (sp->rule != BNS_RULE_BATCH && sp->rule != BNS_RULE_FEATURE) return BNS_ERR_RULE;
+    if (!(mix >= 0.f && mix <= 1.f)) return BNS_ERR_RULE;
+    bns_status st = make_problem(sh, sp, mp.real);
+    if (st != BNS_OK) return st;
+    mp.virt_rule = *sp;
+    mp.virt_rule.rule = BNS_RULE_VIRTUAL;
+    st = make_problem(sh, &mp.virt_rule, mp.virt);
+    if (st != BNS_OK) return st;
+    mp.off_virt = align_up(mp.real.total);
+    mp.off_vec = mp.off_virt + align_up(mp.virt.total);
+    mp.total = mp.off_vec + align_up(2 * static_cast<size_t>(mp.real.C) * sizeof(float));
+    return BNS_OK;
+}
+
+unsigned per_channel_grid(int C) { return static_cast<unsigned>((C + kThreads - 1) / kThreads); }
+
+bns_status forward_mixed_impl(const MixedProblem& mp, const bns_sampling* sp, const void* x, const float* gamma,
+                              const float* beta, float eps, float mix, void* y, float* mean, float* invstd,
+                              float* mean_s, float* mean_v, void* ws, cudaStream_t stream) {
+    const Problem& pr = mp.real;
+    const Problem& pv = mp.virt;
+    void* ws_v = static_cast<char*>(ws) + mp.off_virt;
+    float* invstd_s = ws_at<float>(ws, mp.off_vec);
+    float* invstd_v = invstd_s + pr.C;
+    bns_status st = run_statistics(pr, sp, x, eps, mean_s, invstd_s, ws, stream);        // Eq. 3 on the sampled real set
+    if (st != BNS_OK) return st;
+    st = run_statistics(pv, &mp.virt_rule, x, eps, mean_v, invstd_v, ws_v, stream);      // Eq. 3 on the virtual set
+    if (st != BNS_OK) return st;
+    launch(BNS_KERNEL_VECTOR, mix_stats_kernel, per_channel_grid(pr.C), stream, mean_s, invstd_s, mean_v, invstd_v, mix,
+           pr.C, mean, invstd);                                                           // Eq. 4
+    const ColPlan& pl = pr.main_plan;
+    BNS_BY_TYPE_V(pr.dtype, pl.V,
+                  (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pl.grid(), stream, in<T>(x), out<T>(y), gamma,
+                          beta, mean, invstd, RowOrder{RowOrder::kIdentity, pr.N, 0, 0}, pl.nchunks, pl.tiles, pr.HW,
+                          pr.P)));
+    if (sp->yv) {
+        const ColPlan& pq = pv.stat_plan;
+        BNS_BY_TYPE_V(sp->xv_dtype, pq.V,
+                      (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pq.grid(), stream, in<T>(sp->xv),
+                              out<T>(sp->yv), gamma, beta, mean, invstd, RowOrder{RowOrder::kIdentity, pq.rows, 0, 0},
+                              pq.nchunks, pq.tiles, pr.HW, pr.P)));
+    }
+    return last_error();
+}
+
+bns_status backward_mixed_impl(const MixedProblem& mp, const bns_sampling* sp, const void* x, const void* dy,
+                               const float* gamma, const float* mean, const float* invstd, const float* mean_s,
+                               const float* mean_v, float mix, void* dx, float* dgamma, float* dbeta, void* ws,
+                               cudaStream_t stream) {
+    const Problem& pr = mp.real;
+    const Problem& pv = mp.virt;
+    void* ws_v = static_cast<char*>(ws) + mp.off_virt;
+    const ColPlan& pl = pr.main_plan;
+    const ColPlan& pq = pv.stat_plan;
+    GradSink sink{ws_at<float2>(ws, pr.off_bwd), pl.layout(), sp->dyv ? ws_at<float2>(ws_v, pv.off_bwd_v) : nullptr,
+                  pq.layout(), invstd, dgamma, dbeta};
+    // the sums of Eq. 5 over the real batch (and dx without the statistics terms), then over the virtual rows
+    BNS_BY_TYPE_V(pr.dtype, pl.V,
+                  (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, true>, pl.grid(), stream, in<T>(x), in<T>(dy),
+                          out<T>(dx), gamma, mean, invstd, RowOrder{RowOrder::kIdentity, pr.N, 0, 0}, pl.nchunks, pl.tiles,
+                          pr.HW, pr.P, false, sink)));
+    if (sp->dyv)
+        BNS_BY_TYPE_V(sp->xv_dtype, pq.V,
+                      (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, false>, pq.grid(), stream, in<T>(sp->xv),
+                              in<T>(sp->dyv), out<T>(nullptr), gamma, mean, invstd,
+                              RowOrder{RowOrder::kIdentity, pq.rows, 0, 0}, pq.nchunks, pq.tiles, pr.HW, pr.P, true,
+                              sink)));
+    launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pr.C), stream, sink, pr.C, pr.HW);
+    // statistics terms on the sampled real set: share (1-mix) of dl/dE and dl/dVar, spread over s_s
+    // elements, deviations taken about that set's own mean
+    const float w_s = static_cast<float>((1.0 - static_cast<double>(mix)) / pr.s);
+    if (pr.rule == BNS_RULE_BATCH) {
+        const int* list = nullptr;
+        bns_status st = stage_list(pr, sp, ws, stream, &list);
+        if (st != BNS_OK) return st;
+        const ColPlan& ps = pr.stat_plan;
+        BNS_BY_TYPE_V(pr.dtype, ps.V,
+                      (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, ps.grid(), stream, in<T>(x), in<T>(dy),
+                              out<T>(dx), gamma, mean_s, invstd, dgamma, dbeta, w_s, list, pr.begin,
+                              RowOrder{RowOrder::kIdentity, ps.rows, 0, 0}, ps.nchunks, ps.tiles, pr.HW, pr.P)));
+    } else {
+        unsigned* status;
+        bns_status st = clear_status(pr, ws, stream, &status);
+        if (st != BNS_OK) return st;
+        const PatchPlan& pp = pr.patch_plan;
+        BNS_BY_TYPE(pr.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, patch_fixup_kernel<T>, pp.grid(), stream, in<T>(x), in<T>(dy),
+                                      out<T>(dx), gamma, mean_s, invstd, dgamma, dbeta, w_s, pr.patch, pr.N, pr.C, pr.H,
+                                      pr.W, pp.nchunks, pp.tiles, status)));
+    }
+    // and on the virtual samples: share mix, spread over s_v elements, about the virtual mean
+    if (sp->dxv) {
+        const float w_v = static_cast<float>(static_cast<double>(mix) / pv.s);
+        BNS_BY_TYPE_V(sp->xv_dtype, pq.V,
+                      (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pq.grid(), stream, in<T>(sp->xv),
+                              in<T>(sp->dyv), out<T>(sp->dxv), gamma, mean_v, invstd, dgamma, dbeta, w_v,
+                              static_cast<const int*>(nullptr), 0, RowOrder{RowOrder::kIdentity, pq.rows, 0, 0},
+                              pq.nchunks, pq.tiles, pr.HW, pr.P)));
+    }
+    return last_error();
+}
+
 bns_sampling full_rule() {
     bns_sampling sp;
     std::memset(&sp, 0, sizeof(sp));
@@ -738,8 +850,80 @@ const char* bns_kernel_name(int kernel_kind) {
     case BNS_KERNEL_MASK: return "selection_mask_kernel";
     case BNS_KERNEL_DIRECT_MOMENTS: return "direct_moments_kernel";
     case BNS_KERNEL_DIRECT_FIXUP: return "direct_finalize_fixup_kernel";
+    case BNS_KERNEL_VECTOR: return "per-channel vector kernels";
     }
     return "unknown";
+}
+
+// ---------------------------------------------------------------------------------------- Eq. 4 and Appendix D
+size_t bns_workspace_bytes_mixed(const bns_shape* shape, const bns_sampling* sampling) {
+    MixedProblem mp;
+    if (make_mixed(shape, sampling, 0.5f, mp) != BNS_OK) return 0;
+    return mp.total;
+}
+
+bns_status bns_forward_mixed(const bns_shape* shape, const void* x, const float* gamma, const float* beta, float eps,
+                             float mix, const bns_sampling* sampling, void* y, float* mean, float* invstd, float* mean_s,
+                             float* mean_v, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    MixedProblem mp;
+    bns_status st = make_mixed(shape, sampling, mix, mp);
+    if (st != BNS_OK) return st;
+    if (!x || !gamma || !beta || !y || !mean || !invstd || !mean_s || !mean_v) return BNS_ERR_NULL;
+    if (!(eps > 0.f)) return BNS_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(y)) return BNS_ERR_ALIGN;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) || workspace_bytes < mp.total)
+        return BNS_ERR_WORKSPACE;
+    return forward_mixed_impl(mp, sampling, x, gamma, beta, eps, mix, y, mean, invstd, mean_s, mean_v, workspace,
+                              static_cast<cudaStream_t>(cuda_stream));
+}
+
+bns_status bns_backward_mixed(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
+                              const float* mean, const float* invstd, const float* mean_s, const float* mean_v, float mix,
+                              const bns_sampling* sampling, void* dx, float* dgamma, float* dbeta, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
+    MixedProblem mp;
+    bns_status st = make_mixed(shape, sampling, mix, mp);
+    if (st != BNS_OK) return st;
+    if (!x || !dy || !gamma || !mean || !invstd || !mean_s || !mean_v || !dx || !dgamma || !dbeta) return BNS_ERR_NULL;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dx)) return BNS_ERR_ALIGN;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) || workspace_bytes < mp.total)
+        return BNS_ERR_WORKSPACE;
+    return backward_mixed_impl(mp, sampling, x, dy, gamma, mean, invstd, mean_s, mean_v, mix, dx, dgamma, dbeta, workspace,
+                               static_cast<cudaStream_t>(cuda_stream));
+}
+
+bns_status bns_update_moving_average(int C, const float* mean, const float* invstd, float eps, float alpha,
+                                     int first_iteration, float* mean_ma, float* var_ma, void* cuda_stream) {
+    if (C <= 0 || !(eps > 0.f)) return BNS_ERR_SHAPE;
+    if (!(alpha >= 0.f && alpha <= 1.f)) return BNS_ERR_RULE;
+    if (!mean || !invstd || !mean_ma || !var_ma) return BNS_ERR_NULL;
+    launch(BNS_KERNEL_VECTOR, moving_average_kernel, per_channel_grid(C), static_cast<cudaStream_t>(cuda_stream), mean,
+           invstd, eps, alpha, first_iteration ? 1 : 0, C, mean_ma, var_ma);
+    return last_error();
+}
+
+bns_status bns_inference_forward(const bns_shape* shape, const void* x, const float* gamma, const float* beta, float eps,
+                                 const float* mean_ma, const float* var_ma, void* y, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+    bns_sampling sp = full_rule();
+    Problem pb;
+    bns_status st = make_problem(shape, &sp, pb);
+    if (st != BNS_OK) return st;
+    if (!x || !gamma || !beta || !mean_ma || !var_ma || !y) return BNS_ERR_NULL;
+    if (!(eps > 0.f)) return BNS_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(y)) return BNS_ERR_ALIGN;
+    st = check_workspace(pb, workspace, workspace_bytes);
+    if (st != BNS_OK) return st;
+    if (pb.total - pb.off_stats < static_cast<size_t>(pb.C) * sizeof(float)) return BNS_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    float* invstd = ws_at<float>(workspace, pb.off_stats);
+    launch(BNS_KERNEL_VECTOR, invstd_from_var_kernel, per_channel_grid(pb.C), stream, var_ma, eps, pb.C, invstd);
+    const ColPlan& pl = pb.main_plan;
+    BNS_BY_TYPE_V(pb.dtype, pl.V,
+                  (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pl.grid(), stream, in<T>(x), out<T>(y), gamma,
+                          beta, mean_ma, invstd, RowOrder{RowOrder::kIdentity, pb.N, 0, 0}, pl.nchunks, pl.tiles, pb.HW,
+                          pb.P)));
+    return last_error();
 }
 
 // ---------------------------------------------------------------------------------------- no-allocation forward

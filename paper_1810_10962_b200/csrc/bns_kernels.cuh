@@ -918,6 +918,45 @@ direct_finalize_fixup_kernel(const typename T::storage* __restrict__ src, const 
     }
 }
 
+// ------------------------------------------------------------------------------------ per-channel vector kernels
+// Eq. 4: statistics mixed from the virtual samples (v) and the sampled real set (s) with weight b on
+// the virtual side.  With Var + eps = b (Var_v + eps) + (1-b) (Var_s + eps) the mixed invstd follows
+// from the two invstd without ever forming a variance (no cancellation against eps).
+__global__ void __launch_bounds__(kThreads)
+mix_stats_kernel(const float* __restrict__ mean_s, const float* __restrict__ invstd_s, const float* __restrict__ mean_v,
+                 const float* __restrict__ invstd_v, float b, int C, float* __restrict__ mean, float* __restrict__ invstd) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x * kThreads + threadIdx.x;
+    if (c >= C) return;
+    const float is_s = invstd_s[c], is_v = invstd_v[c];
+    mean[c] = b * mean_v[c] + (1.0f - b) * mean_s[c];
+    invstd[c] = 1.0f / sqrtf(b / (is_v * is_v) + (1.0f - b) / (is_s * is_s));
+}
+
+// Eq. 8: moving average of E and Var; the batch variance is recovered from invstd = (Var + eps)^-1/2.
+__global__ void __launch_bounds__(kThreads)
+moving_average_kernel(const float* __restrict__ mean, const float* __restrict__ invstd, float eps, float alpha, int first,
+                      int C, float* __restrict__ mean_ma, float* __restrict__ var_ma) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x * kThreads + threadIdx.x;
+    if (c >= C) return;
+    const float is = invstd[c];
+    const float E = mean[c], Var = fmaxf(1.0f / (is * is) - eps, 0.f);
+    mean_ma[c] = first ? E : alpha * E + (1.0f - alpha) * mean_ma[c];
+    var_ma[c] = first ? Var : alpha * Var + (1.0f - alpha) * var_ma[c];
+}
+
+// invstd = (Var + eps)^-1/2 from a recorded variance (validation-time forward).
+__global__ void __launch_bounds__(kThreads)
+invstd_from_var_kernel(const float* __restrict__ var, float eps, int C, float* __restrict__ invstd) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x * kThreads + threadIdx.x;
+    if (c < C) invstd[c] = 1.0f / sqrtf(var[c] + eps);
+}
+
 // ------------------------------------------------------------------------------------ selection mask (test aid)
 __global__ void __launch_bounds__(kThreads)
 selection_mask_kernel(uint8_t* __restrict__ mask, int rule, const int* __restrict__ list, int begin, int count,

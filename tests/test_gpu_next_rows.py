@@ -1,0 +1,93 @@
+"""GPU parity for the rows beyond the basic path: VDN combined with a sampling rule (Eq. 4), the moving
+average of the statistics (Eq. 8) and the validation-time forward (Appendix D)."""
+import numpy as np
+import pytest
+
+import bns_inputs as I
+import oracle as O
+from helpers import _to_device, _to_host, close_bf16, close_f32, gpu_sampling, make_case
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("rule,kw", [
+    ("batch", dict(k=3, contiguous=False)), ("batch", dict(k=8)), ("feature", dict(ph=3, pw=3, offset_mode=0)),
+    ("feature", dict(ph=2, pw=5, offset_mode=2)),
+])
+@pytest.mark.parametrize("dtype,dims", [("f32", (40, 24, 20, 20)), ("bf16", (32, 48, 14, 14)), ("f32", (9, 5, 7, 7))])
+@pytest.mark.parametrize("mix,with_dyv", [(0.5, True), (0.25, False)])
+def test_mixed_statistics_forward_backward(rule, kw, dtype, dims, mix, with_dyv):
+    import torch
+    from paper_1810_10962_b200 import bns
+    case = make_case(*dims, rule, seed=93, dtype=dtype, **kw)
+    N, C, H, W = dims
+    xv_np = I.virtual_samples(2, C, H, W, 93)
+    dyv_np = I.upstream_gradient(xv_np.shape, 93, I.TAG_DYV) if with_dyv else None
+    x, dy = _to_device(case.x, dtype), _to_device(case.dy, dtype)
+    gamma, beta = torch.from_numpy(case.gamma).cuda(), torch.from_numpy(case.beta).cuda()
+    xv = torch.from_numpy(xv_np).cuda()
+    dyv = torch.from_numpy(dyv_np).cuda() if with_dyv else None
+    sp = gpu_sampling(case).with_virtual(xv, yv=torch.empty_like(xv), dyv=dyv, dxv=torch.empty_like(xv))
+    y, mean, invstd, mean_s, mean_v = bns.forward_mixed(x, gamma, beta, case.eps, mix, sp)
+    dx, dgamma, dbeta = bns.backward_mixed(x, dy, gamma, mean, invstd, mean_s, mean_v, mix, sp)
+    torch.cuda.synchronize()
+    osp = case.oracle_sampling()
+    f = O.forward_mixed(case.x, xv_np, case.gamma, case.beta, case.eps, mix, osp)
+    b = O.backward_mixed(case.x, xv_np, case.dy, dyv_np, case.gamma, f, case.eps, mix, osp)
+    tensor_close = close_f32 if dtype == "f32" else close_bf16
+    close_f32(mean.cpu().numpy(), f.mean, "mean")
+    close_f32(invstd.cpu().numpy(), f.invstd, "invstd")
+    close_f32(mean_s.cpu().numpy(), f.mean_s, "mean_s")
+    close_f32(mean_v.cpu().numpy(), f.mean_v, "mean_v")
+    tensor_close(_to_host(y), f.y, "y")
+    close_f32(sp.yv.cpu().numpy(), f.yv, "yv")
+    tensor_close(_to_host(dx), b.dx, "dx")
+    close_f32(sp.dxv.cpu().numpy(), b.dxv, "dxv")
+    close_f32(dgamma.cpu().numpy(), b.dgamma, "dgamma")
+    close_f32(dbeta.cpu().numpy(), b.dbeta, "dbeta")
+
+
+def test_mixed_rejects_other_rules_and_weights():
+    import ctypes
+    import torch
+    from paper_1810_10962_b200 import bns
+    x = torch.zeros(4, 4, 8, 8, device="cuda")
+    xv = torch.zeros(2, 4, 8, 8, device="cuda")
+    g = torch.ones(4, device="cuda")
+    with pytest.raises(bns.BnsError):
+        bns.forward_mixed(x, g, g, 1e-5, 0.5, bns.Sampling.virtual(xv))            # needs BATCH or FEATURE
+    sp = bns.Sampling.batch(np.array([0, 1], np.int32)).with_virtual(xv)
+    with pytest.raises(bns.BnsError):
+        bns.forward_mixed(x, g, g, 1e-5, 1.5, sp, workspace=torch.empty(1 << 20, dtype=torch.uint8, device="cuda"))
+
+
+def test_moving_average_and_inference_forward():
+    import torch
+    from paper_1810_10962_b200 import bns
+    N, C, H, W = 32, 24, 10, 10
+    gamma_np, beta_np = I.affine_parameters(C, 94)
+    gamma, beta = torch.from_numpy(gamma_np).cuda(), torch.from_numpy(beta_np).cuda()
+    mean_ma = torch.zeros(C, device="cuda")
+    var_ma = torch.zeros(C, device="cuda")
+    o_mean = o_var = None
+    alpha = 0.7
+    for it in range(4):                       # four training iterations with Batch Sampling, different batches
+        x_np = I.correlated_activations(N, C, H, W, 940 + it)
+        idx = I.batch_sample_indices(N, 4, 940 + it, contiguous=True)
+        x = torch.from_numpy(x_np).cuda()
+        _, mean, invstd = bns.forward(x, gamma, beta, 1e-5, bns.Sampling.batch(idx))
+        bns.update_moving_average(mean, invstd, 1e-5, alpha, it == 0, mean_ma, var_ma)
+        f = O.forward(x_np, gamma_np, beta_np, 1e-5, O.Sampling.batch(idx), want_y=False)
+        o_mean = O.moving_average(f.mean, o_mean, alpha, it == 0)
+        o_var = O.moving_average(f.var, o_var, alpha, it == 0)
+    torch.cuda.synchronize()
+    close_f32(mean_ma.cpu().numpy(), o_mean, "mean_ma")
+    close_f32(var_ma.cpu().numpy(), o_var, "var_ma")
+    for dtype in ("f32", "bf16"):
+        xe_np = I.correlated_activations(N, C, H, W, 949)
+        if dtype == "bf16":
+            xe_np = I.round_to_bf16(xe_np)
+        y = bns.inference_forward(_to_device(xe_np, dtype), gamma, beta, 1e-5, mean_ma, var_ma)
+        want = O.inference_forward(xe_np, gamma_np, beta_np, 1e-5, mean_ma.cpu().numpy().astype(np.float64),
+                                   var_ma.cpu().numpy().astype(np.float64))
+        (close_f32 if dtype == "f32" else close_bf16)(_to_host(y), want, f"inference y {dtype}")
