@@ -237,3 +237,34 @@ def test_small_sampled_sets_both_paths(rule, kw, dtype):
             compare(case, run_gpu(case))
     finally:
         bns.set_tuning("direct_max", 8192)
+
+
+# ----------------------------------------------------------------------------- seeded random sweep
+def _random_specs(count, seed):
+    rng = np.random.default_rng(seed)
+    specs = []
+    for i in range(count):
+        N = int(rng.integers(1, 40))
+        C = int(rng.integers(1, 70))
+        H = int(rng.integers(1, 20))
+        W = int(rng.integers(1, 20))
+        rule = ["batch", "feature", "virtual", "full"][i % 4]
+        dtype = "bf16" if rng.random() < 0.4 else "f32"
+        kw = {}
+        if rule == "batch":
+            kw = dict(k=int(rng.integers(1, N + 1)), contiguous=bool(rng.random() < 0.5))
+        elif rule == "feature":
+            kw = dict(ph=int(rng.integers(1, H + 1)), pw=int(rng.integers(1, W + 1)), offset_mode=int(rng.integers(0, 3)))
+        elif rule == "virtual":
+            kw = dict(nv=int(rng.integers(1, 4)), xv_dtype=dtype if rng.random() < 0.5 else "f32",
+                      with_dyv=bool(rng.random() < 0.5))
+        specs.append((N, C, H, W, rule, dtype, kw, 1000 + i))
+    return specs
+
+
+@pytest.mark.parametrize("spec", _random_specs(48, 2024), ids=lambda s: f"{s[4]}-{s[5]}-{s[0]}x{s[1]}x{s[2]}x{s[3]}")
+def test_random_shapes_and_rules(spec):
+    """Shapes nobody tuned for: odd sizes, one sample, one channel, 1x1 maps, patches of any size."""
+    N, C, H, W, rule, dtype, kw, seed = spec
+    case = make_case(N, C, H, W, rule, seed=seed, dtype=dtype, generator="tiny", **kw)
+    compare(case, run_gpu(case))
