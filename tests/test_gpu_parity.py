@@ -268,3 +268,11 @@ def test_random_shapes_and_rules(spec):
     N, C, H, W, rule, dtype, kw, seed = spec
     case = make_case(N, C, H, W, rule, seed=seed, dtype=dtype, generator="tiny", **kw)
     compare(case, run_gpu(case))
+
+
+@pytest.mark.parametrize("ph,pw,mode", [(1, 1, 0), (1, 1, 2), (2, 2, 1), (1, 3, 0), (2, 4, 2), (1, 8, 0)])
+@pytest.mark.parametrize("dtype,dims", [("bf16", (70, 37, 7, 9)), ("f32", (33, 130, 14, 14)), ("f32", (5, 3, 4, 8))])
+def test_small_patches(ph, pw, mode, dtype, dims):
+    """Patches of a few elements: every map contributes one short row segment, channels far apart."""
+    case = make_case(*dims, "feature", seed=88, dtype=dtype, generator="tiny", ph=ph, pw=pw, offset_mode=mode)
+    compare(case, run_gpu(case))
