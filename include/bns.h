@@ -172,6 +172,41 @@ bns_status bns_inference_forward(const bns_shape* shape, const void* x, const fl
                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Statistics shared by several GPUs (Sec. 4.3 "Micro-BN": Sync-BN with Feature or Batch Sampling).
+ * Each rank holds its own slice of the batch; the sampled statistics are those of the union of the
+ * ranks' sampled sets, so the result equals one big batch normalised with Eq. 1/3 and Eq. 5/6.  The
+ * exchange itself (an all-gather of 3C floats forward, an all-reduce of 2C floats backward) is the
+ * caller's, e.g. NCCL through torch.distributed; these calls are the per-rank pieces around it:
+ *
+ *   bns_sync_local_moments   this rank's sampled set -> moments[3][C] = (count, mean, M2) rows
+ *   (all-gather the 3C floats of every rank into [ranks][3][C])
+ *   bns_sync_merge_moments   merges the ranks' rows in rank order (same bits on every rank) -> mean, invstd
+ *   bns_sync_normalize       Eq. 1 on this rank's x with the shared statistics
+ *   bns_sync_backward_sums   sums[2][C] = (sum dy, sum dy xhat) over this rank's elements, and
+ *                            dx = gamma invstd dy for every element (lower branch of Eq. 6);
+ *                            the two rows are also this rank's share of dbeta and dgamma
+ *   (all-reduce the 2C floats)
+ *   bns_sync_backward_apply  upper branch of Eq. 6 on this rank's sampled elements with the summed
+ *                            rows and sampled_total = the number of sampled points per channel over
+ *                            all ranks
+ * rule may be FULL, BATCH or FEATURE (VIRTUAL: feed the virtual samples to one rank as a BATCH rule
+ * over them).  Workspace as for bns_forward with the same shape and rule (FULL for _backward_sums).
+ */
+bns_status bns_sync_local_moments(const bns_shape* shape, const void* x, const bns_sampling* sampling, float eps,
+                                  float* moments, void* workspace, size_t workspace_bytes, void* cuda_stream);
+bns_status bns_sync_merge_moments(int C, int ranks, const float* moments, float eps, float* mean, float* invstd,
+                                  void* cuda_stream);
+bns_status bns_sync_normalize(const bns_shape* shape, const void* x, const float* gamma, const float* beta,
+                              const float* mean, const float* invstd, void* y, void* cuda_stream);
+bns_status bns_sync_backward_sums(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
+                                  const float* mean, const float* invstd, void* dx, float* sums,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
+                                   const float* mean, const float* invstd, const bns_sampling* sampling,
+                                   const float* sums, double sampled_total, void* dx,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * bns_forward for callers that cannot provide scratch memory.  (The paper has no counterpart; this
  * is a packaging variant of bns_forward: same kernels, same results.)
  *

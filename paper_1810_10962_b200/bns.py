@@ -35,6 +35,8 @@ EXPORTS = [
     "bns_set_tuning",
     "bns_workspace_bytes_mixed", "bns_forward_mixed", "bns_backward_mixed", "bns_update_moving_average",
     "bns_inference_forward",
+    "bns_sync_local_moments", "bns_sync_merge_moments", "bns_sync_normalize", "bns_sync_backward_sums",
+    "bns_sync_backward_apply",
 ]
 
 
@@ -119,6 +121,16 @@ def load():
     lib.bns_update_moving_average.argtypes = [ctypes.c_int, vp, vp, fl, fl, ctypes.c_int, vp, vp, vp]
     lib.bns_inference_forward.restype = ctypes.c_int
     lib.bns_inference_forward.argtypes = [shp, vp, vp, vp, fl, vp, vp, vp, vp, sz, vp]
+    lib.bns_sync_local_moments.restype = ctypes.c_int
+    lib.bns_sync_local_moments.argtypes = [shp, vp, smp, fl, vp, vp, sz, vp]
+    lib.bns_sync_merge_moments.restype = ctypes.c_int
+    lib.bns_sync_merge_moments.argtypes = [ctypes.c_int, ctypes.c_int, vp, fl, vp, vp, vp]
+    lib.bns_sync_normalize.restype = ctypes.c_int
+    lib.bns_sync_normalize.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp]
+    lib.bns_sync_backward_sums.restype = ctypes.c_int
+    lib.bns_sync_backward_sums.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.bns_sync_backward_apply.restype = ctypes.c_int
+    lib.bns_sync_backward_apply.argtypes = [shp, vp, vp, vp, vp, vp, smp, vp, ctypes.c_double, vp, vp, sz, vp]
     lib.bns_set_tuning.restype = ctypes.c_int
     lib.bns_set_tuning.argtypes = [ctypes.c_char_p, ctypes.c_int]
     _lib = lib
@@ -438,6 +450,60 @@ def inference_forward(x, gamma, beta, eps, mean_ma, var_ma, y=None, workspace=No
                                       _vec(mean_ma, C), _vec(var_ma, C), _dev(y), wp, wn, _stream())
     _check(st, "bns_inference_forward")
     return y
+
+
+# ----------------------------------------------------------------------------- statistics shared by several GPUs
+def sync_local_moments(x, sampling: Sampling, eps, workspace=None):
+    """bns_sync_local_moments: float32 [3, C] = (count, mean, M2) of this rank's sampled set."""
+    sh, sp = _shape(x), sampling._c()
+    moments = torch.empty(3, x.shape[1], dtype=torch.float32, device=x.device)
+    ws, wp, wn = _workspace(x, sampling, workspace)
+    _check(load().bns_sync_local_moments(ctypes.byref(sh), _dev(x), ctypes.byref(sp), float(eps), moments.data_ptr(),
+                                         wp, wn, _stream()), "bns_sync_local_moments")
+    return moments
+
+
+def sync_merge_moments(gathered, eps):
+    """bns_sync_merge_moments on a [ranks, 3, C] tensor (an all-gather result): returns (mean, invstd)."""
+    R, three, C = gathered.shape
+    assert three == 3 and gathered.dtype == torch.float32
+    mean, invstd = (torch.empty(C, dtype=torch.float32, device=gathered.device) for _ in range(2))
+    _check(load().bns_sync_merge_moments(C, R, _dev(gathered), float(eps), mean.data_ptr(), invstd.data_ptr(),
+                                         _stream()), "bns_sync_merge_moments")
+    return mean, invstd
+
+
+def sync_normalize(x, gamma, beta, mean, invstd, y=None):
+    sh = _shape(x)
+    C = x.shape[1]
+    y = torch.empty_like(x) if y is None else y
+    _check(load().bns_sync_normalize(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), _vec(mean, C),
+                                     _vec(invstd, C), _dev(y), _stream()), "bns_sync_normalize")
+    return y
+
+
+def sync_backward_sums(x, dy, gamma, mean, invstd, dx=None, workspace=None):
+    """bns_sync_backward_sums: returns (dx without the statistics terms, sums float32 [2, C])."""
+    sh = _shape(x)
+    C = x.shape[1]
+    dx = torch.empty_like(x) if dx is None else dx
+    sums = torch.empty(2, C, dtype=torch.float32, device=x.device)
+    ws, wp, wn = _workspace(x, Sampling.full(), workspace)
+    _check(load().bns_sync_backward_sums(ctypes.byref(sh), _dev(x), _dev(dy), _vec(gamma, C), _vec(mean, C),
+                                         _vec(invstd, C), _dev(dx), sums.data_ptr(), wp, wn, _stream()),
+           "bns_sync_backward_sums")
+    return dx, sums
+
+
+def sync_backward_apply(x, dy, gamma, mean, invstd, sampling: Sampling, sums, sampled_total, dx, workspace=None):
+    """bns_sync_backward_apply: adds the statistics terms to dx on this rank's sampled elements."""
+    sh, sp = _shape(x), sampling._c()
+    C = x.shape[1]
+    ws, wp, wn = _workspace(x, sampling, workspace)
+    _check(load().bns_sync_backward_apply(ctypes.byref(sh), _dev(x), _dev(dy), _vec(gamma, C), _vec(mean, C),
+                                          _vec(invstd, C), ctypes.byref(sp), _dev(sums), float(sampled_total), _dev(dx),
+                                          wp, wn, _stream()), "bns_sync_backward_apply")
+    return dx
 
 
 # ----------------------------------------------------------------------------- host-buffer step

@@ -926,6 +926,118 @@ bns_status bns_inference_forward(const bns_shape* shape, const void* x, const fl
     return last_error();
 }
 
+// ---------------------------------------------------------------------------------------- statistics shared by several GPUs
+bns_status bns_sync_local_moments(const bns_shape* shape, const void* x, const bns_sampling* sampling, float eps,
+                                  float* moments, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    Problem pb;
+    bns_status st = make_problem(shape, sampling, pb);
+    if (st != BNS_OK) return st;
+    if (pb.rule == BNS_RULE_VIRTUAL) return BNS_ERR_RULE;
+    if (!x || !moments) return BNS_ERR_NULL;
+    if (!(eps > 0.f)) return BNS_ERR_SHAPE;
+    if (!aligned16(x)) return BNS_ERR_ALIGN;
+    st = check_workspace(pb, workspace, workspace_bytes);
+    if (st != BNS_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = run_statistics(pb, sampling, x, eps, moments + pb.C, moments + 2 * pb.C, workspace, stream);
+    if (st != BNS_OK) return st;
+    launch(BNS_KERNEL_VECTOR, moments_rows_kernel, per_channel_grid(pb.C), stream, moments, static_cast<float>(pb.s), eps,
+           pb.C);
+    return last_error();
+}
+
+bns_status bns_sync_merge_moments(int C, int ranks, const float* moments, float eps, float* mean, float* invstd,
+                                  void* cuda_stream) {
+    if (C <= 0 || ranks <= 0 || !(eps > 0.f)) return BNS_ERR_SHAPE;
+    if (!moments || !mean || !invstd) return BNS_ERR_NULL;
+    launch(BNS_KERNEL_VECTOR, merge_rank_moments_kernel, per_channel_grid(C), static_cast<cudaStream_t>(cuda_stream),
+           moments, ranks, C, eps, mean, invstd);
+    return last_error();
+}
+
+bns_status bns_sync_normalize(const bns_shape* shape, const void* x, const float* gamma, const float* beta,
+                              const float* mean, const float* invstd, void* y, void* cuda_stream) {
+    bns_sampling sp = full_rule();
+    Problem pb;
+    bns_status st = make_problem(shape, &sp, pb);
+    if (st != BNS_OK) return st;
+    if (!x || !gamma || !beta || !mean || !invstd || !y) return BNS_ERR_NULL;
+    if (!aligned16(x) || !aligned16(y)) return BNS_ERR_ALIGN;
+    const ColPlan& pl = pb.main_plan;
+    BNS_BY_TYPE_V(pb.dtype, pl.V,
+                  (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pl.grid(), static_cast<cudaStream_t>(cuda_stream),
+                          in<T>(x), out<T>(y), gamma, beta, mean, invstd, RowOrder{RowOrder::kIdentity, pb.N, 0, 0},
+                          pl.nchunks, pl.tiles, pb.HW, pb.P)));
+    return last_error();
+}
+
+bns_status bns_sync_backward_sums(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
+                                  const float* mean, const float* invstd, void* dx, float* sums, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream) {
+    bns_sampling sp = full_rule();
+    Problem pb;
+    bns_status st = make_problem(shape, &sp, pb);
+    if (st != BNS_OK) return st;
+    if (!x || !dy || !gamma || !mean || !invstd || !dx || !sums) return BNS_ERR_NULL;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dx)) return BNS_ERR_ALIGN;
+    st = check_workspace(pb, workspace, workspace_bytes);
+    if (st != BNS_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const ColPlan& pl = pb.main_plan;
+    // row 0: sum dy (dbeta), row 1: sum dy xhat (dgamma) over this rank's elements
+    GradSink sink{ws_at<float2>(workspace, pb.off_bwd), pl.layout(), nullptr, pl.layout(), invstd, sums + pb.C, sums};
+    BNS_BY_TYPE_V(pb.dtype, pl.V,
+                  (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, true>, pl.grid(), stream, in<T>(x), in<T>(dy),
+                          out<T>(dx), gamma, mean, invstd, RowOrder{RowOrder::kIdentity, pb.N, 0, 0}, pl.nchunks, pl.tiles,
+                          pb.HW, pb.P, false, sink)));
+    launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
+    return last_error();
+}
+
+bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
+                                   const float* mean, const float* invstd, const bns_sampling* sampling,
+                                   const float* sums, double sampled_total, void* dx, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream) {
+    Problem pb;
+    bns_status st = make_problem(shape, sampling, pb);
+    if (st != BNS_OK) return st;
+    if (pb.rule == BNS_RULE_VIRTUAL) return BNS_ERR_RULE;
+    if (!x || !dy || !gamma || !mean || !invstd || !sums || !dx) return BNS_ERR_NULL;
+    if (!(sampled_total >= pb.s)) return BNS_ERR_SHAPE;  // the shared set holds at least this rank's share
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dx)) return BNS_ERR_ALIGN;
+    st = check_workspace(pb, workspace, workspace_bytes);
+    if (st != BNS_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const float* dbeta = sums;
+    const float* dgamma = sums + pb.C;
+    const float inv_s = static_cast<float>(1.0 / sampled_total);
+    const ColPlan& pl = pb.main_plan;
+    const ColPlan& pv = pb.stat_plan;
+    if (pb.rule == BNS_RULE_FULL) {
+        BNS_BY_TYPE_V(pb.dtype, pl.V,
+                      (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pl.grid(), stream, in<T>(x), in<T>(dy),
+                              out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, static_cast<const int*>(nullptr), 0,
+                              RowOrder{RowOrder::kIdentity, pl.rows, 0, 0}, pl.nchunks, pl.tiles, pb.HW, pb.P)));
+    } else if (pb.rule == BNS_RULE_BATCH) {
+        const int* list = nullptr;
+        st = stage_list(pb, sampling, workspace, stream, &list);
+        if (st != BNS_OK) return st;
+        BNS_BY_TYPE_V(pb.dtype, pv.V,
+                      (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(x), in<T>(dy),
+                              out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, list, pb.begin,
+                              RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P)));
+    } else {
+        unsigned* status;
+        st = clear_status(pb, workspace, stream, &status);
+        if (st != BNS_OK) return st;
+        const PatchPlan& pp = pb.patch_plan;
+        BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, patch_fixup_kernel<T>, pp.grid(), stream, in<T>(x), in<T>(dy),
+                                      out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, pb.patch, pb.N, pb.C, pb.H,
+                                      pb.W, pp.nchunks, pp.tiles, status)));
+    }
+    return last_error();
+}
+
 // ---------------------------------------------------------------------------------------- no-allocation forward
 // Scratch for bns_forward_static: a fixed array in device memory that is part of the loaded library
 // image, so a caller that has no way to obtain device memory of its own can still run the forward.

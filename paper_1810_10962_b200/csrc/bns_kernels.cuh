@@ -957,6 +957,37 @@ invstd_from_var_kernel(const float* __restrict__ var, float eps, int C, float* _
     if (c < C) invstd[c] = 1.0f / sqrtf(var[c] + eps);
 }
 
+// ------------------------------------------------------------------------------------ statistics shared by several GPUs
+// A rank's sampled statistics as (count, mean, M2) rows of C floats, the form in which ranks exchange
+// them; rows 1 and 2 arrive holding mean and invstd and row 2 is turned into M2 = count (1/invstd^2 - eps).
+__global__ void __launch_bounds__(kThreads)
+moments_rows_kernel(float* __restrict__ rows, float count, float eps, int C) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x * kThreads + threadIdx.x;
+    if (c >= C) return;
+    const float is = rows[2 * C + c];
+    rows[c] = count;
+    rows[2 * C + c] = count * fmaxf(1.0f / (is * is) - eps, 0.f);
+}
+
+// Merges the (count, mean, M2) rows of R ranks (rank-major: [R][3][C]) in rank order.
+__global__ void __launch_bounds__(kThreads)
+merge_rank_moments_kernel(const float* __restrict__ rows, int R, int C, float eps, float* __restrict__ mean,
+                          float* __restrict__ invstd) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x * kThreads + threadIdx.x;
+    if (c >= C) return;
+    Moments acc = {0.f, 0.f, 0.f};
+    for (int r = 0; r < R; ++r) {
+        const float* q = rows + static_cast<size_t>(r) * 3 * C;
+        acc = merge(acc, Moments{q[c], q[C + c], q[2 * C + c]});
+    }
+    mean[c] = acc.mean;
+    invstd[c] = 1.0f / sqrtf(acc.m2 / acc.cnt + eps);
+}
+
 // ------------------------------------------------------------------------------------ selection mask (test aid)
 __global__ void __launch_bounds__(kThreads)
 selection_mask_kernel(uint8_t* __restrict__ mask, int rule, const int* __restrict__ list, int begin, int count,

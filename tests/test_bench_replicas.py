@@ -63,3 +63,30 @@ def test_workloads_match_the_configured_shapes():
     bs = r18[0]
     assert bs.algorithmic_bytes() == int(round((5 + 4 * 32 / 256) * bs.elems * 4)) + 32 * 64
     assert [(l.C, l.H) for l in bench.workload_layers("cifar")] == I.cifar_resnet_layers()
+
+
+def _exchange_rank(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_1810_10962_b200 import sync
+    rows = torch.full((3, 4), float(rank + 1))
+    gathered = sync.all_gather_rows(rows)
+    sums = sync.all_reduce_rows(torch.full((2, 4), float(rank + 1)))
+    out[rank] = (gathered.tolist(), sums.tolist(), rows.tolist())
+    dist.destroy_process_group()
+
+
+@pytest.mark.timeout(120)
+def test_shared_statistics_exchange_between_two_ranks():
+    """The only traffic of the shared-statistics path: an all-gather of the (count, mean, M2) rows in rank
+    order and a sum of the backward rows (gloo, CPU tensors; the arithmetic around it runs on the GPU)."""
+    world, port = 2, _free_port()
+    with mp.Manager() as manager:
+        out = manager.dict()
+        mp.spawn(_exchange_rank, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    for rank in range(world):
+        gathered, sums, rows = res[rank]
+        assert gathered == [[[1.0] * 4] * 3, [[2.0] * 4] * 3]       # rank-major, same on every rank
+        assert sums == [[3.0] * 4] * 2
+        assert rows == [[float(rank + 1)] * 4] * 3                  # the input is left alone

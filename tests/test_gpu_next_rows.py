@@ -91,3 +91,53 @@ def test_moving_average_and_inference_forward():
         want = O.inference_forward(xe_np, gamma_np, beta_np, 1e-5, mean_ma.cpu().numpy().astype(np.float64),
                                    var_ma.cpu().numpy().astype(np.float64))
         (close_f32 if dtype == "f32" else close_bf16)(_to_host(y), want, f"inference y {dtype}")
+
+
+@pytest.mark.parametrize("rule", ["batch", "feature", "full"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("ranks", [2, 3])
+def test_statistics_shared_by_several_ranks_equal_one_big_batch(rule, dtype, ranks):
+    """Sync-BN with sampling: the batch is split over `ranks` slices, each slice goes through the per-rank
+    calls, the exchanges are a stack (all-gather) and a sum (all-reduce) on the one GPU, and the result
+    must be the oracle's for the whole batch with the union of the ranks' sampled sets."""
+    import torch
+    from paper_1810_10962_b200 import bns
+    from helpers import quantise
+    n_local, C, H, W = 8, 20, 12, 12
+    N = n_local * ranks
+    x_np = quantise(I.correlated_activations(N, C, H, W, 95), dtype)
+    dy_np = quantise(I.upstream_gradient(x_np.shape, 95), dtype)
+    gamma_np, beta_np = I.affine_parameters(C, 95)
+    gamma, beta = torch.from_numpy(gamma_np).cuda(), torch.from_numpy(beta_np).cuda()
+    eps = 1e-5
+    local_idx = [np.array([1 + r, 5], np.int32) for r in range(ranks)]          # each rank samples two of its slices
+    offsets = np.array([[3, 2]], np.int32)
+    if rule == "batch":
+        osp = O.Sampling.batch(np.concatenate([idx + r * n_local for r, idx in enumerate(local_idx)]))
+        sps = [bns.Sampling.batch(idx) for idx in local_idx]
+    elif rule == "feature":
+        osp = O.Sampling.feature(4, 5, offsets)
+        sps = [bns.Sampling.feature(4, 5, offsets) for _ in range(ranks)]
+    else:
+        osp = O.Sampling.full()
+        sps = [bns.Sampling.full() for _ in range(ranks)]
+    s_total = O.sample_count(N, H, W, osp)
+    xs = [_to_device(x_np[r * n_local:(r + 1) * n_local], dtype) for r in range(ranks)]
+    dys = [_to_device(dy_np[r * n_local:(r + 1) * n_local], dtype) for r in range(ranks)]
+    gathered = torch.stack([bns.sync_local_moments(xs[r], sps[r], eps) for r in range(ranks)])   # "all-gather"
+    mean, invstd = bns.sync_merge_moments(gathered, eps)
+    ys = [bns.sync_normalize(xs[r], gamma, beta, mean, invstd) for r in range(ranks)]
+    partial = [bns.sync_backward_sums(xs[r], dys[r], gamma, mean, invstd) for r in range(ranks)]
+    sums = torch.stack([p[1] for p in partial]).sum(dim=0)                                        # "all-reduce"
+    dxs = [bns.sync_backward_apply(xs[r], dys[r], gamma, mean, invstd, sps[r], sums, s_total, partial[r][0])
+           for r in range(ranks)]
+    torch.cuda.synchronize()
+    f = O.forward(x_np, gamma_np, beta_np, eps, osp)
+    b = O.backward(x_np, dy_np, gamma_np, f.mean, f.var, eps, osp)
+    tensor_close = close_f32 if dtype == "f32" else close_bf16
+    close_f32(mean.cpu().numpy(), f.mean, "mean")
+    close_f32(invstd.cpu().numpy(), f.invstd, "invstd")
+    tensor_close(np.concatenate([_to_host(t) for t in ys]), f.y, "y")
+    tensor_close(np.concatenate([_to_host(t) for t in dxs]), b.dx, "dx")
+    close_f32(sums[0].cpu().numpy(), b.dbeta, "dbeta")
+    close_f32(sums[1].cpu().numpy(), b.dgamma, "dgamma")
