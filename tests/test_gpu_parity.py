@@ -276,3 +276,39 @@ def test_small_patches(ph, pw, mode, dtype, dims):
     """Patches of a few elements: every map contributes one short row segment, channels far apart."""
     case = make_case(*dims, "feature", seed=88, dtype=dtype, generator="tiny", ph=ph, pw=pw, offset_mode=mode)
     compare(case, run_gpu(case))
+
+
+@pytest.mark.parametrize("rule,kw", [("batch", dict(k=4)), ("feature", dict(ph=3, pw=3)), ("full", dict())])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_host_buffer_entry_point(rule, kw, dtype):
+    """bns_forward_backward_host: pinned host tensors in, pinned host tensors out, copies on the stream."""
+    import torch
+    from paper_1810_10962_b200 import bns
+    from helpers import run_oracle, close_f32, close_bf16, _to_host
+    import bns_inputs as I
+    case = make_case(20, 12, 10, 10, rule, seed=89, dtype=dtype, **kw)
+    dt = torch.float32 if dtype == "f32" else torch.bfloat16
+
+    def pin(a):
+        t = torch.from_numpy(a)
+        if dtype == "bf16":
+            t = torch.from_numpy(I.f32_to_bf16_bits(a).view(np.int16)).view(torch.bfloat16)
+        return t.pin_memory()
+
+    x, dy = pin(case.x), pin(case.dy)
+    y, dx = torch.empty_like(x).pin_memory(), torch.empty_like(x).pin_memory()
+    C = case.x.shape[1]
+    mean, invstd, dgamma, dbeta = (torch.empty(C, dtype=torch.float32).pin_memory() for _ in range(4))
+    gamma, beta = torch.from_numpy(case.gamma).pin_memory(), torch.from_numpy(case.beta).pin_memory()
+    sp = gpu_sampling(case)
+    arena = torch.empty(bns.host_arena_bytes(tuple(case.x.shape), dt, sp), dtype=torch.uint8, device="cuda")
+    bns.forward_backward_host(x, dy, gamma, beta, case.eps, sp, y, dx, mean, invstd, dgamma, dbeta, arena)
+    torch.cuda.synchronize()
+    f, b = run_oracle(case)
+    tensor_close = close_f32 if dtype == "f32" else close_bf16
+    close_f32(mean.numpy(), f.mean, "mean")
+    close_f32(invstd.numpy(), f.invstd, "invstd")
+    tensor_close(_to_host(y), f.y, "y")
+    tensor_close(_to_host(dx), b.dx, "dx")
+    close_f32(dgamma.numpy(), b.dgamma, "dgamma")
+    close_f32(dbeta.numpy(), b.dbeta, "dbeta")
