@@ -66,7 +66,10 @@ typedef struct {
     /* BATCH */
     int k;                      /* number of sampled samples, 1..N                                */
     const int32_t* sample_idx;  /* HOST, k distinct values in [0,N), any order; copied during the */
-                                /* call, so it may be reused as soon as the call returns          */
+                                /* call, so it may be reused as soon as the call returns.  A list */
+                                /* begin..begin+k-1 (the paper's rule) needs no copy; any other   */
+                                /* list is sent with cudaMemcpyAsync, so pin it if the stream is  */
+                                /* being captured into a graph                                    */
     /* FEATURE */
     int ph, pw;                 /* patch size, 1..H and 1..W                                      */
     int offset_mode;            /* bns_offset_mode                                                */

@@ -283,7 +283,8 @@ bool g_l2_order = true;
 int g_direct_max = 8192;  // sampled elements per channel up to which one block per channel handles the sampled set  // order rows so that a kernel re-reads what the previous one left in L2
 
 template <typename... KArgs, typename... Args>
-void launch(int kind, void (*kernel)(KArgs...), unsigned grid, cudaStream_t s, Args&&... args) {
+void launch_with(bool early_scheduling, int kind, void (*kernel)(KArgs...), unsigned grid, cudaStream_t s,
+                 Args&&... args) {
     LaunchScope scope(kind, s);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -294,8 +295,21 @@ void launch(int kind, void (*kernel)(KArgs...), unsigned grid, cudaStream_t s, A
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = g_pdl ? 1 : 0;
+    cfg.numAttrs = (g_pdl && early_scheduling) ? 1 : 0;
     cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// Normal launch of this library: the kernel may be scheduled while its predecessor drains.
+template <typename... KArgs, typename... Args>
+void launch(int kind, void (*kernel)(KArgs...), unsigned grid, cudaStream_t s, Args&&... args) {
+    launch_with(true, kind, kernel, grid, s, static_cast<Args&&>(args)...);
+}
+
+// For a kernel that touches its inputs before its dependency wait and is the first kernel of a call:
+// whatever precedes it in the stream may have produced those inputs, so it must not start early.
+template <typename... KArgs, typename... Args>
+void launch_after_predecessor(int kind, void (*kernel)(KArgs...), unsigned grid, cudaStream_t s, Args&&... args) {
+    launch_with(false, kind, kernel, grid, s, static_cast<Args&&>(args)...);
 }
 
 #define BNS_BY_TYPE_V(dtype, V_, CALL)                   \
@@ -965,8 +979,9 @@ bns_status bns_sync_normalize(const bns_shape* shape, const void* x, const float
     if (!aligned16(x) || !aligned16(y)) return BNS_ERR_ALIGN;
     const ColPlan& pl = pb.main_plan;
     BNS_BY_TYPE_V(pb.dtype, pl.V,
-                  (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pl.grid(), static_cast<cudaStream_t>(cuda_stream),
-                          in<T>(x), out<T>(y), gamma, beta, mean, invstd, RowOrder{RowOrder::kIdentity, pb.N, 0, 0},
+                  (launch_after_predecessor(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pl.grid(),
+                                            static_cast<cudaStream_t>(cuda_stream), in<T>(x), out<T>(y), gamma, beta, mean,
+                                            invstd, RowOrder{RowOrder::kIdentity, pb.N, 0, 0},
                           pl.nchunks, pl.tiles, pb.HW, pb.P)));
     return last_error();
 }
