@@ -439,6 +439,15 @@ def run_ours(args):
             lms, _ = time_steps(torch, dist, runner(d.step)[0], args.steps, args.warmup, local, world)
             per_layer[d.layer.name]["full_bn_ms"] = round(lms, 5)
             per_layer[d.layer.name]["speedup_vs_full_bn"] = round(lms / per_layer[d.layer.name]["ms"], 4)
+        # the paper's estimation errors (Sec. 5.1, "Correlation Analysis"): E_mu = ||mu_s - mu||_2 and
+        # E_sigma = ||sigma_s - sigma||_2 between the sampled statistics and those of the whole batch,
+        # from the vectors the two forward calls above left behind (diagnostic; synthetic activations)
+        torch.cuda.synchronize()
+        for d, f in zip(dev, full):
+            sigma_s, sigma = 1.0 / d.invstd.double(), 1.0 / f.invstd.double()     # sqrt(var + eps) each
+            per_layer[d.layer.name]["estimation_error"] = {
+                "E_mu": round(float((d.mean.double() - f.mean.double()).norm()), 6),
+                "E_sigma": round(float((sigma_s - sigma).norm()), 6), "channels": d.layer.C}
 
     # ---- roofline of the dominant kernel: backward pass 1 reads dy and x and writes dx (3 E b per launch)
     roofline = None
