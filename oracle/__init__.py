@@ -290,3 +290,38 @@ def inference_forward(x, gamma, beta, eps, E_ma, Var_ma) -> np.ndarray:
     _library().oracle_inference_forward(N, C, H, W, _ptr(x), _ptr(gamma), _ptr(beta), ctypes.c_double(eps), _ptr(E_ma),
                                         _ptr(Var_ma), _ptr(y))
     return y
+
+
+# ----------------------------------------------------------------------------- BN followed by a residual add and ReLU
+# Not an equation of the paper: the step that follows every BN layer of the ResNets it trains
+# (y = max(0, BN(x) + r)).  Stated here by composing the pinned BN forward/backward above with the
+# definition of the rectifier, so that a fused GPU version has something to be compared with.
+@dataclass
+class ForwardAct:
+    y: np.ndarray        # max(0, z)
+    z: np.ndarray        # BN(x) + residual, before the rectifier
+    mean: np.ndarray
+    var: np.ndarray
+    invstd: np.ndarray
+
+
+def forward_relu(x, residual, gamma, beta, eps, sp: Sampling, channels=None) -> ForwardAct:
+    assert sp.rule != RULE_VIRTUAL
+    f = forward(x, gamma, beta, eps, sp, channels=channels)
+    z = f.y
+    if residual is not None:
+        r = _f32(residual).astype(np.float64)
+        z = z + (r if channels is None else r[:, np.asarray(channels)])
+    return ForwardAct(np.maximum(z, 0.0), z, f.mean, f.var, f.invstd)
+
+
+def backward_relu(x, dy, gamma, fwd: ForwardAct, eps, sp: Sampling, channels=None):
+    """Returns (Backward for the BN part with the rectifier's gradient applied, dresidual = dy * [z > 0])."""
+    dyf = _f32(dy)
+    sel = slice(None) if channels is None else np.asarray(channels)
+    g_sel = np.where(fwd.z > 0.0, dyf[:, sel].astype(np.float64), 0.0)
+    # the C oracle takes float32 gradients: g is dy or 0, both exactly representable
+    g = np.zeros_like(dyf)
+    g[:, sel] = g_sel.astype(np.float32)
+    b = backward(x, g, gamma, fwd.mean, fwd.var, eps, sp, channels=channels)
+    return b, g_sel

@@ -177,3 +177,33 @@ def test_inference_forward_is_library_eval_batch_norm():
     t = lambda a: torch.tensor(np.asarray(a), dtype=torch.float64)
     want = torch.nn.functional.batch_norm(t(x), t(E_ma), t(Var_ma), t(gamma), t(beta), training=False, eps=EPS)
     np.testing.assert_allclose(y, want.numpy(), rtol=1e-13, atol=1e-14)
+
+
+# --------------------------------------------------------------------------- BN + residual + ReLU
+@pytest.mark.parametrize("with_residual", [True, False])
+def test_relu_composition_matches_autograd(with_residual):
+    x, dy, gamma, beta, xv, dyv = small(46)
+    N, C, H, W = x.shape
+    res = I.upstream_gradient(x.shape, 46, I.TAG_XV) if with_residual else None
+    for name, sp in list(rules(N, C, H, W, 46).items()) + [("full", O.Sampling.full())]:
+        f = O.forward_relu(x, res, gamma, beta, EPS, sp)
+        b, dres = O.backward_relu(x, dy, gamma, f, EPS, sp)
+        t = lambda a: torch.tensor(a, dtype=torch.float64)
+        xt, gt, bt = t(x).requires_grad_(), t(gamma).requires_grad_(), t(beta).requires_grad_()
+        rt = t(res).requires_grad_() if with_residual else None
+        mt = t(O.selection_mask(N, C, H, W, sp))
+        sh = (1, -1, 1, 1)
+        s = mt.sum(dim=(0, 2, 3))
+        mean = (xt * mt).sum(dim=(0, 2, 3)) / s
+        var = (((xt - mean.view(sh)) ** 2) * mt).sum(dim=(0, 2, 3)) / s
+        z = gt.view(sh) * (xt - mean.view(sh)) / torch.sqrt(var.view(sh) + EPS) + bt.view(sh)
+        if with_residual:
+            z = z + rt
+        y = torch.relu(z)
+        (y * t(dy)).sum().backward()
+        np.testing.assert_allclose(f.y, y.detach().numpy(), rtol=1e-12, atol=1e-13, err_msg=name)
+        np.testing.assert_allclose(b.dx, xt.grad.numpy(), rtol=1e-10, atol=1e-12, err_msg=name)
+        np.testing.assert_allclose(b.dgamma, gt.grad.numpy(), rtol=1e-11, atol=1e-12, err_msg=name)
+        np.testing.assert_allclose(b.dbeta, bt.grad.numpy(), rtol=1e-11, atol=1e-12, err_msg=name)
+        if with_residual:
+            np.testing.assert_allclose(dres, rt.grad.numpy(), rtol=0, atol=0, err_msg=name)
