@@ -65,7 +65,7 @@ class Layer:
             return m
         if self.rule == "batch":
             return self.kw["k"] * self.H * self.W
-        if self.rule in ("feature", "mixed"):
+        if self.rule in ("feature", "mixed", "relu"):
             return self.N * self.kw["ph"] * self.kw["pw"]
         return self.kw["nv"] * self.H * self.W
 
@@ -75,6 +75,11 @@ class Layer:
         vec = 16 * C
         if self.rule == "full":
             return 8 * E * b + 2 * vec
+        if self.rule == "relu":
+            # forward reads x, residual, the patches and writes y; backward reads x, residual, dy, writes dx and
+            # dresidual; the fix-up reads x, residual, dy on S and writes dx there
+            r = self.sampled_per_channel() / (self.N * self.H * self.W)
+            return int(round((8 + 5 * r) * E * b)) + 2 * vec
         if self.rule == "mixed":
             ev = self.kw["nv"] * C * self.H * self.W * 4      # xv is fp32: statistics, yv, and dxv as for VDN
             r = self.sampled_per_channel() / (self.N * self.H * self.W)
@@ -107,6 +112,9 @@ def workload_layers(name):
     if name == "fs_vdn":
         # the paper's most accurate variant (Table 2, "FS+VDN"): Eq. 4 with a patch and two virtual samples
         return [Layer("fs8x8_vdn2", 256, 64, 56, 56, "f32", "mixed", ph=8, pw=8, nv=2, mix=0.5)]
+    if name == "fs_relu":
+        # the block a ResNet actually runs: BN (Feature Sampling) + residual add + ReLU, fused
+        return [Layer("fs8x8_res_relu", 256, 64, 56, 56, "f32", "relu", ph=8, pw=8)]
     if name == "tiny":
         return [Layer("bs2", 8, 16, 8, 8, "f32", "batch", k=2)]
     raise SystemExit(f"unknown workload {name}")
@@ -125,7 +133,7 @@ def selected_layers(args):
 
 
 def layer_seed(workload, index):
-    return 1810 + 100 * (["tiny", "cifar", "resnet18_stage1", "vdn", "resnet50", "fs_vdn"].index(workload) + 1) + index
+    return 1810 + 100 * (["tiny", "cifar", "resnet18_stage1", "vdn", "resnet50", "fs_vdn", "fs_relu"].index(workload) + 1) + index
 
 
 def host_inputs(layer: Layer, seed):
@@ -147,6 +155,9 @@ def host_inputs(layer: Layer, seed):
     elif layer.rule == "mixed":
         extra["offsets"] = I.patch_offsets(N, C, H, W, layer.kw["ph"], layer.kw["pw"], I.OFFSETS_SHARED, seed)
         extra["xv"] = I.virtual_samples(layer.kw["nv"], C, H, W, seed)
+    elif layer.rule == "relu":
+        extra["offsets"] = I.patch_offsets(N, C, H, W, layer.kw["ph"], layer.kw["pw"], I.OFFSETS_SHARED, seed)
+        extra["residual"] = I.upstream_gradient(x.shape, seed, I.TAG_XV)
     return dict(x=x, dy=dy, gamma=gamma, beta=beta, **extra)
 
 
@@ -219,6 +230,7 @@ class DeviceLayer:
         self.layer, self.bns, self.torch = layer, bns, torch
         self.full = full_bn or layer.rule == "full"
         self.mixed = layer.rule == "mixed" and not self.full
+        self.relu = layer.rule == "relu"      # the full-BN comparison runs through the same fused kernels
         dt = torch.float32 if layer.dtype == "f32" else torch.bfloat16
 
         def dev(a):
@@ -231,6 +243,12 @@ class DeviceLayer:
         self.gamma, self.beta = torch.from_numpy(host["gamma"]).cuda(), torch.from_numpy(host["beta"]).cuda()
         C = layer.C
         self.mean, self.invstd, self.dgamma, self.dbeta = (torch.empty(C, device="cuda") for _ in range(4))
+        if self.relu:
+            self.sp = (bns.Sampling.full() if self.full
+                       else bns.Sampling.feature(layer.kw["ph"], layer.kw["pw"], host["offsets"]))
+            self.residual = dev(host["residual"])
+            self.ws = bns.new_workspace(x, self.sp)
+            return
         if self.full:
             self.sp = bns.Sampling.full()
         elif layer.rule == "batch":
@@ -254,6 +272,12 @@ class DeviceLayer:
                       for sx, sdy, sy, sdx in self.sets]
 
     def step(self, i):
+        if self.relu:
+            x, dy, _, _ = self.sets[i % len(self.sets)]
+            b = self.bns
+            _, mean, invstd = b.forward_relu(x, self.residual, self.gamma, self.beta, EPS, self.sp, workspace=self.ws)
+            b.backward_relu(x, self.residual, dy, self.gamma, self.beta, mean, invstd, self.sp, workspace=self.ws)
+            return
         if self.mixed:
             x, dy, y, dx = self.sets[i % len(self.sets)]
             b, mix = self.bns, self.layer.kw["mix"]
@@ -432,7 +456,9 @@ def run_ours(args):
     full_info = None
     if full:
         fms, _ = time_steps(torch, dist, runner(full_step)[0], args.steps, args.warmup, local, world)
-        fbytes = sum(l.count * (8 * l.elems * l.ebytes + 32 * l.C) for l in layers)
+        # full BN: 3 passes forward + 5 backward; with the fused residual + ReLU 4 + 9 (residual read three times,
+        # dresidual written, the second backward pass re-reads x, residual and dy)
+        fbytes = sum(l.count * ((13 if l.rule == "relu" else 8) * l.elems * l.ebytes + 32 * l.C) for l in layers)
         full_info = {"ms_per_step": round(fms, 5), "gbps": round(fbytes / fms / 1e6, 1), "algorithmic_bytes": fbytes,
                      "speedup_sampled_vs_full": round(fms / ms_plain, 4)}
         for d in full:
@@ -444,6 +470,8 @@ def run_ours(args):
         # from the vectors the two forward calls above left behind (diagnostic; synthetic activations)
         torch.cuda.synchronize()
         for d, f in zip(dev, full):
+            if d.relu:
+                continue                      # that path keeps its statistics in tensors of its own
             sigma_s, sigma = 1.0 / d.invstd.double(), 1.0 / f.invstd.double()     # sqrt(var + eps) each
             per_layer[d.layer.name]["estimation_error"] = {
                 "E_mu": round(float((d.mean.double() - f.mean.double()).norm()), 6),
@@ -503,7 +531,7 @@ def run_e2e(torch, bns, layers, hosts, steps):
     """Same metric through bns_forward_backward_host: pinned host tensors in, pinned host tensors out."""
     items, h2d, d2h = [], 0, 0
     for l, h in zip(layers, hosts):
-        if l.rule in ("virtual", "mixed"):
+        if l.rule in ("virtual", "mixed", "relu"):
             return None      # the host entry point keeps xv on the device; not measured end to end
         dt = torch.float32 if l.dtype == "f32" else torch.bfloat16
         pin = lambda a: torch.from_numpy(a).to(dt).pin_memory()
@@ -560,6 +588,12 @@ def oracle_sample(layers, hosts, seconds):
         else:
             sp = O.Sampling.full()
         ch = np.asarray(channels, dtype=np.int32)
+        if l.rule == "relu":
+            sp = O.Sampling.feature(l.kw["ph"], l.kw["pw"], h["offsets"])
+            t0 = time.perf_counter()
+            f = O.forward_relu(h["x"], h["residual"], h["gamma"], h["beta"], EPS, sp, channels=ch)
+            O.backward_relu(h["x"], h["dy"], h["gamma"], f, EPS, sp, channels=ch)
+            return time.perf_counter() - t0
         if l.rule == "mixed":
             sp = O.Sampling.feature(l.kw["ph"], l.kw["pw"], h["offsets"])
             t0 = time.perf_counter()
@@ -636,7 +670,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="resnet18_stage1",
-                    choices=["resnet18_stage1", "cifar", "vdn", "resnet50", "fs_vdn", "tiny"])
+                    choices=["resnet18_stage1", "cifar", "vdn", "resnet50", "fs_vdn", "fs_relu", "tiny"])
     ap.add_argument("--only", default=None, help="comma-separated layer names: run just these layers of the workload")
     ap.add_argument("--tune", action="append", default=[], metavar="NAME=VALUE",
                     help="launch-shape knob of the library (bns_set_tuning), e.g. --tune pdl=0")

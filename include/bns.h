@@ -210,6 +210,25 @@ bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const 
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * BN with sampled statistics followed by a residual add and a ReLU, fused:
+ *   forward   y = max(0, gamma xhat + beta + residual)
+ *   backward  g = dy where gamma xhat + beta + residual > 0, else 0;  dresidual = g;  then bns_backward
+ *             with g in place of dy (sums, dx, statistics terms on S).
+ * This is not an equation of the paper: it is the step that follows every BN layer of the residual
+ * networks it trains (Table 1); fusing it saves writing and re-reading the pre-activation tensor.  The
+ * mask is recomputed from x and residual, nothing is stored for it, so the backward call needs beta and
+ * the same residual.  residual and dresidual may be NULL (plain BN + ReLU; dresidual may also be NULL
+ * when only dx is wanted).  rule FULL, BATCH or FEATURE; workspace as for bns_forward.
+ */
+bns_status bns_forward_relu(const bns_shape* shape, const void* x, const void* residual, const float* gamma,
+                            const float* beta, float eps, const bns_sampling* sampling, void* y, float* mean,
+                            float* invstd, void* workspace, size_t workspace_bytes, void* cuda_stream);
+bns_status bns_backward_relu(const bns_shape* shape, const void* x, const void* residual, const void* dy,
+                             const float* gamma, const float* beta, const float* mean, const float* invstd,
+                             const bns_sampling* sampling, void* dx, void* dresidual, float* dgamma, float* dbeta,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * bns_forward for callers that cannot provide scratch memory.  (The paper has no counterpart; this
  * is a packaging variant of bns_forward: same kernels, same results.)
  *

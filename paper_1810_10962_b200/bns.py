@@ -37,6 +37,7 @@ EXPORTS = [
     "bns_inference_forward",
     "bns_sync_local_moments", "bns_sync_merge_moments", "bns_sync_normalize", "bns_sync_backward_sums",
     "bns_sync_backward_apply",
+    "bns_forward_relu", "bns_backward_relu",
 ]
 
 
@@ -131,6 +132,10 @@ def load():
     lib.bns_sync_backward_sums.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.bns_sync_backward_apply.restype = ctypes.c_int
     lib.bns_sync_backward_apply.argtypes = [shp, vp, vp, vp, vp, vp, smp, vp, ctypes.c_double, vp, vp, sz, vp]
+    lib.bns_forward_relu.restype = ctypes.c_int
+    lib.bns_forward_relu.argtypes = [shp, vp, vp, vp, vp, fl, smp, vp, vp, vp, vp, sz, vp]
+    lib.bns_backward_relu.restype = ctypes.c_int
+    lib.bns_backward_relu.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, smp, vp, vp, vp, vp, vp, sz, vp]
     lib.bns_set_tuning.restype = ctypes.c_int
     lib.bns_set_tuning.argtypes = [ctypes.c_char_p, ctypes.c_int]
     _lib = lib
@@ -504,6 +509,37 @@ def sync_backward_apply(x, dy, gamma, mean, invstd, sampling: Sampling, sums, sa
                                           _vec(invstd, C), ctypes.byref(sp), _dev(sums), float(sampled_total), _dev(dx),
                                           wp, wn, _stream()), "bns_sync_backward_apply")
     return dx
+
+
+# ----------------------------------------------------------------------------- BN + residual add + ReLU
+def forward_relu(x, residual, gamma, beta, eps, sampling: Sampling, workspace=None):
+    """bns_forward_relu: returns (y, mean, invstd) with y = max(0, BN(x) + residual); residual may be None."""
+    sh, sp = _shape(x), sampling._c()
+    C = x.shape[1]
+    y = torch.empty_like(x)
+    mean, invstd = (torch.empty(C, dtype=torch.float32, device=x.device) for _ in range(2))
+    ws, wp, wn = _workspace(x, sampling, workspace)
+    st = load().bns_forward_relu(ctypes.byref(sh), _dev(x), None if residual is None else _dev(residual), _vec(gamma, C),
+                                 _vec(beta, C), float(eps), ctypes.byref(sp), _dev(y), _vec(mean, C), _vec(invstd, C),
+                                 wp, wn, _stream())
+    _check(st, "bns_forward_relu")
+    return y, mean, invstd
+
+
+def backward_relu(x, residual, dy, gamma, beta, mean, invstd, sampling: Sampling, workspace=None):
+    """bns_backward_relu: returns (dx, dresidual or None, dgamma, dbeta)."""
+    sh, sp = _shape(x), sampling._c()
+    C = x.shape[1]
+    dx = torch.empty_like(x)
+    dres = None if residual is None else torch.empty_like(x)
+    dgamma, dbeta = (torch.empty(C, dtype=torch.float32, device=x.device) for _ in range(2))
+    ws, wp, wn = _workspace(x, sampling, workspace)
+    st = load().bns_backward_relu(ctypes.byref(sh), _dev(x), None if residual is None else _dev(residual), _dev(dy),
+                                  _vec(gamma, C), _vec(beta, C), _vec(mean, C), _vec(invstd, C), ctypes.byref(sp),
+                                  _dev(dx), None if dres is None else _dev(dres), _vec(dgamma, C), _vec(dbeta, C), wp, wn,
+                                  _stream())
+    _check(st, "bns_backward_relu")
+    return dx, dres, dgamma, dbeta
 
 
 # ----------------------------------------------------------------------------- host-buffer step

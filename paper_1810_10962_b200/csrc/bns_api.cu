@@ -1053,6 +1053,74 @@ bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const 
     return last_error();
 }
 
+// ---------------------------------------------------------------------------------------- BN + residual add + ReLU
+bns_status bns_forward_relu(const bns_shape* shape, const void* x, const void* residual, const float* gamma,
+                            const float* beta, float eps, const bns_sampling* sampling, void* y, float* mean,
+                            float* invstd, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    Problem pb;
+    bns_status st = make_problem(shape, sampling, pb);
+    if (st != BNS_OK) return st;
+    if (pb.rule == BNS_RULE_VIRTUAL) return BNS_ERR_RULE;
+    if (!x || !gamma || !beta || !y || !mean || !invstd) return BNS_ERR_NULL;
+    if (!(eps > 0.f)) return BNS_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(residual)) return BNS_ERR_ALIGN;
+    st = check_workspace(pb, workspace, workspace_bytes);
+    if (st != BNS_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = run_statistics(pb, sampling, x, eps, mean, invstd, workspace, stream);
+    if (st != BNS_OK) return st;
+    const ColPlan& pl = pb.main_plan;
+    BNS_BY_TYPE_V(pb.dtype, pl.V,
+                  (launch(BNS_KERNEL_NORMALIZE, act_normalize_kernel<T, V>, pl.grid(), stream, in<T>(x), in<T>(residual),
+                          out<T>(y), gamma, beta, mean, invstd, pl.rows, pl.nchunks, pl.tiles, pb.HW, pb.P)));
+    return last_error();
+}
+
+bns_status bns_backward_relu(const bns_shape* shape, const void* x, const void* residual, const void* dy,
+                             const float* gamma, const float* beta, const float* mean, const float* invstd,
+                             const bns_sampling* sampling, void* dx, void* dresidual, float* dgamma, float* dbeta,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    Problem pb;
+    bns_status st = make_problem(shape, sampling, pb);
+    if (st != BNS_OK) return st;
+    if (pb.rule == BNS_RULE_VIRTUAL) return BNS_ERR_RULE;
+    if (!x || !dy || !gamma || !beta || !mean || !invstd || !dx || !dgamma || !dbeta) return BNS_ERR_NULL;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dx) || !aligned16(residual) || !aligned16(dresidual))
+        return BNS_ERR_ALIGN;
+    st = check_workspace(pb, workspace, workspace_bytes);
+    if (st != BNS_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const ColPlan& pl = pb.main_plan;
+    const ColPlan& pv = pb.stat_plan;
+    GradSink sink{ws_at<float2>(workspace, pb.off_bwd), pl.layout(), nullptr, pl.layout(), invstd, dgamma, dbeta};
+    BNS_BY_TYPE_V(pb.dtype, pl.V,
+                  (launch(BNS_KERNEL_BWD_REDUCE, act_bwd_reduce_kernel<T, V>, pl.grid(), stream, in<T>(x), in<T>(residual),
+                          in<T>(dy), out<T>(dx), out<T>(dresidual), gamma, beta, mean, invstd, pl.rows, pl.nchunks,
+                          pl.tiles, pb.HW, pb.P, sink)));
+    launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
+    const float inv_s = static_cast<float>(1.0 / pb.s);
+    if (pb.rule == BNS_RULE_FEATURE) {
+        unsigned* status;
+        st = clear_status(pb, workspace, stream, &status);
+        if (st != BNS_OK) return st;
+        const PatchPlan& pp = pb.patch_plan;
+        BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, act_patch_fixup_kernel<T>, pp.grid(), stream, in<T>(x),
+                                      in<T>(residual), in<T>(dy), out<T>(dx), gamma, beta, mean, invstd, dgamma, dbeta,
+                                      inv_s, pb.patch, pb.N, pb.C, pb.H, pb.W, pp.nchunks, pp.tiles, status)));
+    } else {
+        const int* list = nullptr;
+        st = stage_list(pb, sampling, workspace, stream, &list);
+        if (st != BNS_OK) return st;
+        const ColPlan& pf = pb.rule == BNS_RULE_FULL ? pl : pv;
+        BNS_BY_TYPE_V(pb.dtype, pf.V,
+                      (launch(BNS_KERNEL_COL_FIXUP, act_col_fixup_kernel<T, V>, pf.grid(), stream, in<T>(x),
+                              in<T>(residual), in<T>(dy), out<T>(dx), gamma, beta, mean, invstd, dgamma, dbeta, inv_s,
+                              list, pb.rule == BNS_RULE_BATCH ? pb.begin : 0, pf.rows, pf.nchunks, pf.tiles, pb.HW,
+                              pb.P)));
+    }
+    return last_error();
+}
+
 // ---------------------------------------------------------------------------------------- no-allocation forward
 // Scratch for bns_forward_static: a fixed array in device memory that is part of the loaded library
 // image, so a caller that has no way to obtain device memory of its own can still run the forward.

@@ -988,6 +988,195 @@ merge_rank_moments_kernel(const float* __restrict__ rows, int R, int C, float ep
     invstd[c] = 1.0f / sqrtf(acc.m2 / acc.cnt + eps);
 }
 
+// ------------------------------------------------------------------------------------ BN + residual add + ReLU
+// The step that follows a BN layer in a residual network, fused so that the pre-activation tensor is
+// never written: forward y = max(0, a x + b + r); backward g = dy where a x + b + r > 0, else 0, and g
+// takes the place of dy everywhere (sums, dx, statistics terms); dr = g.  The mask is recomputed from
+// x (and r) instead of being stored.  r / dr may be NULL.  These kernels mirror col_normalize,
+// col_bwd_reduce, col_fixup and patch_fixup; they are kept apart from them on purpose.
+struct ActCoef {
+    float a, b;  // z = a x + b (+ r)
+};
+
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+act_normalize_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ res,
+                     typename T::storage* __restrict__ y, const float* __restrict__ gamma,
+                     const float* __restrict__ beta, const float* __restrict__ mean, const float* __restrict__ invstd,
+                     int rows, int nchunks, unsigned tiles, int HW, unsigned P) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const unsigned tile = blockIdx.x % tiles;
+    const int ck = static_cast<int>(blockIdx.x / tiles);
+    const unsigned p = (tile * kThreads + threadIdx.x) * V;
+    if (p >= P) return;
+    float a[V], b[V];
+    {
+        int c[V];
+        position_channels<V>(p, HW, c);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            a[j] = gamma[c[j]] * invstd[c[j]];
+            b[j] = fmaf(-mean[c[j]], a[j], beta[c[j]]);
+        }
+    }
+    for (int i = ck; i < rows; i += kUnroll * nchunks) {
+        Vec<T, V> vx[kUnroll], vr[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (i + u * nchunks < rows) {
+                const size_t off = static_cast<size_t>(i + u * nchunks) * P + p;
+                vx[u].load(x + off);
+                if (res) vr[u].load(res + off);
+            }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (i + u * nchunks < rows) {
+#pragma unroll
+                for (int j = 0; j < V; ++j) {
+                    float z = fmaf(a[j], vx[u].get(j), b[j]);
+                    if (res) z += vr[u].get(j);
+                    vx[u].set(j, fmaxf(z, 0.f));
+                }
+                vx[u].store(y + static_cast<size_t>(i + u * nchunks) * P + p);
+            }
+    }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+act_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ res,
+                      const typename T::storage* __restrict__ dy, typename T::storage* __restrict__ dx,
+                      typename T::storage* __restrict__ dres, const float* __restrict__ gamma,
+                      const float* __restrict__ beta, const float* __restrict__ mean, const float* __restrict__ invstd,
+                      int rows, int nchunks, unsigned tiles, int HW, unsigned P, GradSink G) {
+    constexpr unsigned TP = kThreads * V;
+    __shared__ float s_dy[TP];
+    __shared__ float s_dyxc[TP];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const unsigned tile = blockIdx.x % tiles;
+    const int ck = static_cast<int>(blockIdx.x / tiles);
+    const unsigned p = (tile * kThreads + threadIdx.x) * V;
+    float acc_dy[V], acc_dyxc[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc_dy[j] = acc_dyxc[j] = 0.f;
+    if (p < P) {
+        float a[V], b[V], mu[V];
+        {
+            int c[V];
+            position_channels<V>(p, HW, c);
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                mu[j] = mean[c[j]];
+                a[j] = gamma[c[j]] * invstd[c[j]];
+                b[j] = fmaf(-mu[j], a[j], beta[c[j]]);
+            }
+        }
+        for (int i = ck; i < rows; i += nchunks) {
+            const size_t off = static_cast<size_t>(i) * P + p;
+            Vec<T, V> vx, vg, vr;
+            vx.load(x + off);
+            vg.load(dy + off);
+            if (res) vr.load(res + off);
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                const float xv = vx.get(j);
+                float z = fmaf(a[j], xv, b[j]);
+                if (res) z += vr.get(j);
+                const float g = z > 0.f ? vg.get(j) : 0.f;
+                acc_dy[j] += g;
+                acc_dyxc[j] = fmaf(g, xv - mu[j], acc_dyxc[j]);
+                vg.set(j, g);
+                vx.set(j, a[j] * g);
+            }
+            vx.store(dx + off);
+            if (dres) vg.store(dres + off);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        s_dy[threadIdx.x * V + j] = acc_dy[j];
+        s_dyxc[threadIdx.x * V + j] = acc_dyxc[j];
+    }
+    __syncthreads();
+    fold_sums(s_dy, s_dyxc, TileChannels(tile, TP, P, HW), HW,
+              G.partials + (static_cast<size_t>(ck) * tiles + tile) * G.L.max_slots);
+}
+
+// masked gradient of one element: dy where the pre-activation is positive
+__device__ __forceinline__ float act_gradient(float a, float b, float x, float r, float dy) {
+    return fmaf(a, x, b) + r > 0.f ? dy : 0.f;
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+act_col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ res,
+                     const typename T::storage* __restrict__ dy, typename T::storage* __restrict__ dx,
+                     const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
+                     const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
+                     float inv_s, const int* __restrict__ list, int begin, int count, int nchunks, unsigned tiles,
+                     int HW, unsigned P) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const unsigned tile = blockIdx.x % tiles;
+    const int ck = static_cast<int>(blockIdx.x / tiles);
+    const unsigned p = (tile * kThreads + threadIdx.x) * V;
+    if (p >= P) return;
+    FixCoef k[V];
+    float b[V];
+    {
+        int c[V];
+        position_channels<V>(p, HW, c);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            k[j] = fix_coef(gamma[c[j]], mean[c[j]], invstd[c[j]], dgamma[c[j]], dbeta[c[j]], inv_s);
+            b[j] = fmaf(-k[j].mu, k[j].a, beta[c[j]]);
+        }
+    }
+    for (int i = ck; i < count; i += nchunks) {
+        const int n = list ? list[i] : begin + i;
+        const size_t off = static_cast<size_t>(n) * P + p;
+        Vec<T, V> vx, vg, vr;
+        vx.load(x + off);
+        vg.load(dy + off);
+        if (res) vr.load(res + off);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            const float xv = vx.get(j);
+            const float g = act_gradient(k[j].a, b[j], xv, res ? vr.get(j) : 0.f, vg.get(j));
+            vg.set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (xv - k[j].mu));
+        }
+        vg.store(dx + off);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+act_patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ res,
+                       const typename T::storage* __restrict__ dy, typename T::storage* __restrict__ dx,
+                       const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
+                       const float* __restrict__ invstd, const float* __restrict__ dgamma,
+                       const float* __restrict__ dbeta, float inv_s, PatchRule rule, int N, int C, int H, int W,
+                       int nchunks, unsigned tiles, unsigned* status) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const unsigned tile = blockIdx.x % tiles;
+    const int ck = static_cast<int>(blockIdx.x / tiles);
+    const unsigned j = tile * kThreads + threadIdx.x;
+    if (j >= static_cast<unsigned>(C) * rule.ph * rule.pw) return;
+    const PatchThread me(j, rule, H, W);
+    const size_t P = static_cast<size_t>(C) * H * W;
+    const FixCoef k = fix_coef(gamma[me.c], mean[me.c], invstd[me.c], dgamma[me.c], dbeta[me.c], inv_s);
+    const float b = fmaf(-k.mu, k.a, beta[me.c]);
+    for (int n = ck; n < N; n += nchunks) {
+        const size_t at = me.at(rule, n, P, H, W, status);
+        const float xv = to_float<T>(x[at]);
+        const float g = act_gradient(k.a, b, xv, res ? to_float<T>(res[at]) : 0.f, to_float<T>(dy[at]));
+        dx[at] = from_float<T>(fmaf(k.a, g, -k.A) - k.Q * (xv - k.mu));
+    }
+}
+
 // ------------------------------------------------------------------------------------ selection mask (test aid)
 __global__ void __launch_bounds__(kThreads)
 selection_mask_kernel(uint8_t* __restrict__ mask, int rule, const int* __restrict__ list, int begin, int count,

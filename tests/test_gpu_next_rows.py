@@ -141,3 +141,45 @@ def test_statistics_shared_by_several_ranks_equal_one_big_batch(rule, dtype, ran
     tensor_close(np.concatenate([_to_host(t) for t in dxs]), b.dx, "dx")
     close_f32(sums[0].cpu().numpy(), b.dbeta, "dbeta")
     close_f32(sums[1].cpu().numpy(), b.dgamma, "dgamma")
+
+
+@pytest.mark.parametrize("rule,kw", [("batch", dict(k=5, contiguous=False)), ("batch", dict(k=4)),
+                                     ("feature", dict(ph=3, pw=4, offset_mode=0)),
+                                     ("feature", dict(ph=2, pw=2, offset_mode=2)), ("full", dict())])
+@pytest.mark.parametrize("dtype,dims", [("f32", (24, 20, 14, 14)), ("bf16", (16, 24, 7, 7))])
+@pytest.mark.parametrize("with_residual", [True, False])
+def test_fused_residual_relu(rule, kw, dtype, dims, with_residual):
+    """BN + residual + ReLU against the oracle's composition.  The rectifier's mask is a floating-point
+    decision, so the case is drawn (deterministically) with every pre-activation away from zero by more
+    than the two sides' rounding; then the masks agree and everything is compared element by element."""
+    import torch
+    from paper_1810_10962_b200 import bns
+    from helpers import quantise
+    for seed in range(96, 196):
+        case = make_case(*dims, rule, seed=seed, dtype=dtype, **kw)
+        res_np = quantise(I.upstream_gradient(case.x.shape, seed, I.TAG_XV), dtype) if with_residual else None
+        osp = case.oracle_sampling()
+        f = O.forward_relu(case.x, res_np, case.gamma, case.beta, case.eps, osp)
+        if np.abs(f.z).min() > 2e-5:
+            break
+    else:
+        pytest.fail("no seed keeps the pre-activations away from zero")
+    b, dres_want = O.backward_relu(case.x, case.dy, case.gamma, f, case.eps, osp)
+    x, dy = _to_device(case.x, dtype), _to_device(case.dy, dtype)
+    res = _to_device(res_np, dtype) if with_residual else None
+    gamma, beta = torch.from_numpy(case.gamma).cuda(), torch.from_numpy(case.beta).cuda()
+    sp = gpu_sampling(case)
+    y, mean, invstd = bns.forward_relu(x, res, gamma, beta, case.eps, sp)
+    dx, dres, dgamma, dbeta = bns.backward_relu(x, res, dy, gamma, beta, mean, invstd, sp)
+    torch.cuda.synchronize()
+    tensor_close = close_f32 if dtype == "f32" else close_bf16
+    close_f32(mean.cpu().numpy(), f.mean, "mean")
+    close_f32(invstd.cpu().numpy(), f.invstd, "invstd")
+    tensor_close(_to_host(y), f.y, "y")
+    tensor_close(_to_host(dx), b.dx, "dx")
+    close_f32(dgamma.cpu().numpy(), b.dgamma, "dgamma")
+    close_f32(dbeta.cpu().numpy(), b.dbeta, "dbeta")
+    if with_residual:
+        assert np.array_equal(_to_host(dres), dres_want.astype(np.float32))     # dy or 0: bit-exact
+    else:
+        assert dres is None
