@@ -229,6 +229,24 @@ bns_status bns_backward_relu(const bns_shape* shape, const void* x, const void* 
                              void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Channels-last tensors: x, y, dy, dx (and xv, yv, dyv, dxv) are dense [N,H,W,C] - the layout the paper
+ * itself works in (Appendix A: statistics reduce dims 0,1,2 of B in R^{N x H x W x C}).  Same
+ * arithmetic, arguments and results as bns_forward / bns_backward; `shape` still names N, C, H, W.
+ * All rules are supported; Feature Sampling takes a shared or per-sample patch location (a per-map
+ * location would give every channel of a pixel a different patch: BNS_ERR_RULE).  A sampled pixel is a
+ * contiguous vector of C channels in this layout, so the patch passes read whole cache lines.
+ * Workspace: bns_workspace_bytes_nhwc().
+ */
+size_t bns_workspace_bytes_nhwc(const bns_shape* shape, const bns_sampling* sampling);
+bns_status bns_forward_nhwc(const bns_shape* shape, const void* x, const float* gamma, const float* beta,
+                            float eps, const bns_sampling* sampling, void* y, float* mean, float* invstd,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+bns_status bns_backward_nhwc(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
+                             const float* mean, const float* invstd, const bns_sampling* sampling,
+                             void* dx, float* dgamma, float* dbeta,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * bns_forward for callers that cannot provide scratch memory.  (The paper has no counterpart; this
  * is a packaging variant of bns_forward: same kernels, same results.)
  *

@@ -38,6 +38,7 @@ EXPORTS = [
     "bns_sync_local_moments", "bns_sync_merge_moments", "bns_sync_normalize", "bns_sync_backward_sums",
     "bns_sync_backward_apply",
     "bns_forward_relu", "bns_backward_relu",
+    "bns_workspace_bytes_nhwc", "bns_forward_nhwc", "bns_backward_nhwc",
 ]
 
 
@@ -136,6 +137,12 @@ def load():
     lib.bns_forward_relu.argtypes = [shp, vp, vp, vp, vp, fl, smp, vp, vp, vp, vp, sz, vp]
     lib.bns_backward_relu.restype = ctypes.c_int
     lib.bns_backward_relu.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, smp, vp, vp, vp, vp, vp, sz, vp]
+    lib.bns_workspace_bytes_nhwc.restype = sz
+    lib.bns_workspace_bytes_nhwc.argtypes = [shp, smp]
+    lib.bns_forward_nhwc.restype = ctypes.c_int
+    lib.bns_forward_nhwc.argtypes = [shp, vp, vp, vp, fl, smp, vp, vp, vp, vp, sz, vp]
+    lib.bns_backward_nhwc.restype = ctypes.c_int
+    lib.bns_backward_nhwc.argtypes = [shp, vp, vp, vp, vp, vp, smp, vp, vp, vp, vp, sz, vp]
     lib.bns_set_tuning.restype = ctypes.c_int
     lib.bns_set_tuning.argtypes = [ctypes.c_char_p, ctypes.c_int]
     _lib = lib
@@ -540,6 +547,46 @@ def backward_relu(x, residual, dy, gamma, beta, mean, invstd, sampling: Sampling
                                   _stream())
     _check(st, "bns_backward_relu")
     return dx, dres, dgamma, dbeta
+
+
+# ----------------------------------------------------------------------------- channels-last tensors
+def _shape_nhwc(x: torch.Tensor) -> _Shape:
+    if x.dim() != 4:
+        raise TypeError("expected an NHWC tensor")
+    N, H, W, C = x.shape
+    return _Shape(N, C, H, W, _dtype_code(x))
+
+
+def forward_nhwc(x, gamma, beta, eps, sampling: Sampling, workspace=None):
+    """bns_forward_nhwc on a dense [N,H,W,C] tensor (virtual tensors in `sampling` are [nv,H,W,C] too);
+    returns (y, mean, invstd, workspace) - pass the workspace on to backward_nhwc."""
+    sh, sp = _shape_nhwc(x), sampling._c()
+    C = x.shape[3]
+    n = load().bns_workspace_bytes_nhwc(ctypes.byref(sh), ctypes.byref(sp))
+    if n == 0:
+        raise BnsError(-3, "bns_workspace_bytes_nhwc (invalid shape or sampling rule)")
+    if workspace is None:
+        workspace = torch.empty(int(n), dtype=torch.uint8, device=x.device)
+    y = torch.empty_like(x)
+    mean, invstd = (torch.empty(C, dtype=torch.float32, device=x.device) for _ in range(2))
+    st = load().bns_forward_nhwc(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), ctypes.byref(sp),
+                                 _dev(y), _vec(mean, C), _vec(invstd, C), workspace.data_ptr(), workspace.numel(),
+                                 _stream())
+    _check(st, "bns_forward_nhwc")
+    return y, mean, invstd, workspace
+
+
+def backward_nhwc(x, dy, gamma, mean, invstd, sampling: Sampling, workspace):
+    """bns_backward_nhwc: returns (dx, dgamma, dbeta)."""
+    sh, sp = _shape_nhwc(x), sampling._c()
+    C = x.shape[3]
+    dx = torch.empty_like(x)
+    dgamma, dbeta = (torch.empty(C, dtype=torch.float32, device=x.device) for _ in range(2))
+    st = load().bns_backward_nhwc(ctypes.byref(sh), _dev(x), _dev(dy), _vec(gamma, C), _vec(mean, C), _vec(invstd, C),
+                                  ctypes.byref(sp), _dev(dx), _vec(dgamma, C), _vec(dbeta, C), workspace.data_ptr(),
+                                  workspace.numel(), _stream())
+    _check(st, "bns_backward_nhwc")
+    return dx, dgamma, dbeta
 
 
 # ----------------------------------------------------------------------------- host-buffer step

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "bns_kernels.cuh"
+#include "bns_nhwc_kernels.cuh"
 
 namespace {
 
@@ -646,6 +647,209 @@ bns_status backward_mixed_impl(const MixedProblem& mp, const bns_sampling* sp, c
     return last_error();
 }
 
+// ------------------------------------------------------------------------------------ channels-last (NHWC)
+struct NhwcLaunch {
+    NhwcShape shape;
+    dim3 grid;
+    size_t partial_count() const { return static_cast<size_t>(grid.x) * shape.C; }
+    PartialLayout layout() const {  // the NCHW layout with one position per channel and a single tile
+        return PartialLayout{static_cast<int>(grid.x), 1u, 0x7fffffffu, shape.C};
+    }
+};
+
+// Block shape and grid for visiting `total` rows of C channels.
+NhwcLaunch plan_nhwc(int C, int ebytes, long total, bool statistics) {
+    NhwcLaunch l{};
+    int V = 16 / ebytes;
+    while (V > 1 && C % V != 0) V >>= 1;
+    NhwcShape& s = l.shape;
+    s.C = C;
+    s.V_unused = V;
+    s.CV = C / V;
+    s.CW = std::min(s.CV, kThreads);
+    s.RL = kThreads / s.CW;
+    const int gy = (s.CV + s.CW - 1) / s.CW;
+    const long target = std::max(1L, static_cast<long>(statistics ? g_stat_target_blocks : g_target_blocks) / gy);
+    long rpb = std::max<long>(static_cast<long>(s.RL) * kUnroll * 2, (total + target - 1) / target);
+    rpb = (rpb + s.RL - 1) / s.RL * s.RL;
+    s.rows_per_block = static_cast<int>(rpb);
+    l.grid = dim3(static_cast<unsigned>(std::max(1L, (total + rpb - 1) / rpb)), static_cast<unsigned>(gy), 1);
+    return l;
+}
+
+int nhwc_vector(int C, int ebytes) {
+    int V = 16 / ebytes;
+    while (V > 1 && C % V != 0) V >>= 1;
+    return V;
+}
+
+struct NhwcProblem {
+    Problem pb;                  // shape and rule, validated as for NCHW
+    long rows;                   // N*H*W
+    long sampled_rows;           // rows in the sampled set (of x, or of xv for VIRTUAL)
+    NhwcLaunch main, stat, virt; // all rows of x; the sampled rows; all rows of xv
+    size_t off_list, off_stats, off_bwd, off_bwd_v, total;
+};
+
+bns_status make_nhwc(const bns_shape* sh, const bns_sampling* sp, NhwcProblem& np) {
+    bns_status st = make_problem(sh, sp, np.pb);
+    if (st != BNS_OK) return st;
+    const Problem& pb = np.pb;
+    if (pb.rule == BNS_RULE_FEATURE && sp->offset_mode == BNS_OFF_PER_MAP) return BNS_ERR_RULE;  // a row spans all channels
+    np.rows = static_cast<long>(pb.N) * pb.HW;
+    if (np.rows >= 2147483647L) return BNS_ERR_SHAPE;
+    const int eb = elem_bytes(pb.dtype);
+    np.main = plan_nhwc(pb.C, eb, np.rows, false);
+    np.virt = np.main;
+    switch (pb.rule) {
+    case BNS_RULE_FULL: np.sampled_rows = np.rows; break;
+    case BNS_RULE_BATCH: np.sampled_rows = static_cast<long>(pb.count) * pb.HW; break;
+    case BNS_RULE_FEATURE: np.sampled_rows = static_cast<long>(pb.N) * pb.patch.ph * pb.patch.pw; break;
+    default:
+        np.sampled_rows = static_cast<long>(pb.count) * pb.HW;
+        np.virt = plan_nhwc(pb.C, elem_bytes(sp->xv_dtype), np.sampled_rows, false);
+        break;
+    }
+    const int stat_eb = pb.rule == BNS_RULE_VIRTUAL ? elem_bytes(sp->xv_dtype) : eb;
+    np.stat = plan_nhwc(pb.C, stat_eb, np.sampled_rows, pb.rule != BNS_RULE_FULL);
+    size_t off = kHeaderBytes;
+    np.off_list = off;
+    off += align_up(static_cast<size_t>(pb.N) * sizeof(int));
+    np.off_stats = off;
+    off += align_up(np.stat.partial_count() * sizeof(float4));
+    np.off_bwd = off;
+    off += align_up(np.main.partial_count() * sizeof(float2));
+    np.off_bwd_v = off;
+    if (pb.rule == BNS_RULE_VIRTUAL) off += align_up(np.virt.partial_count() * sizeof(float2));
+    np.total = off;
+    return BNS_OK;
+}
+
+// The sampled rows of the real tensor (or, for VIRTUAL, all rows of xv) as a RowSet.
+RowSet nhwc_row_set(const NhwcProblem& np, const int* list) {
+    const Problem& pb = np.pb;
+    RowSet set{};
+    set.total = static_cast<int>(np.sampled_rows);
+    set.HW = pb.HW;
+    set.H = pb.H;
+    set.W = pb.W;
+    set.list = list;
+    set.begin = pb.begin;
+    set.patch = pb.patch;
+    set.mode = pb.rule == BNS_RULE_BATCH ? RowSet::kSamples : pb.rule == BNS_RULE_FEATURE ? RowSet::kPatches : RowSet::kAll;
+    return set;
+}
+
+bns_status nhwc_stage_list(const NhwcProblem& np, const bns_sampling* sp, void* ws, cudaStream_t stream, const int** list) {
+    *list = nullptr;
+    if (np.pb.rule != BNS_RULE_BATCH || np.pb.contiguous) return BNS_OK;
+    int* dev = ws_at<int>(ws, np.off_list);
+    if (cudaMemcpyAsync(dev, sp->sample_idx, sizeof(int) * sp->k, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return BNS_ERR_CUDA;
+    *list = dev;
+    return BNS_OK;
+}
+
+#define BNS_NHWC_BY_TYPE_V(dtype, C_, CALL)                                  \
+    do {                                                                     \
+        const int V_ = nhwc_vector(C_, elem_bytes(dtype));                   \
+        BNS_BY_TYPE_V(dtype, V_, CALL);                                      \
+    } while (0)
+
+template <typename... KArgs, typename... Args>
+void launch_grid(int kind, void (*kernel)(KArgs...), dim3 grid, cudaStream_t s, Args&&... args) {
+    LaunchScope scope(kind, s);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+bns_status forward_nhwc_impl(const NhwcProblem& np, const bns_sampling* sp, const void* x, const float* gamma,
+                             const float* beta, float eps, void* y, float* mean, float* invstd, void* ws,
+                             cudaStream_t stream) {
+    const Problem& pb = np.pb;
+    unsigned* status;
+    bns_status st = clear_status(pb, ws, stream, &status);
+    if (st != BNS_OK) return st;
+    const int* list = nullptr;
+    st = nhwc_stage_list(np, sp, ws, stream, &list);
+    if (st != BNS_OK) return st;
+    const RowSet set = nhwc_row_set(np, list);
+    const bool virt = pb.rule == BNS_RULE_VIRTUAL;
+    const void* data = virt ? sp->xv : x;
+    const int dt = virt ? sp->xv_dtype : pb.dtype;
+    float4* partials = ws_at<float4>(ws, np.off_stats);
+    BNS_NHWC_BY_TYPE_V(dt, pb.C, (launch_grid(BNS_KERNEL_COL_MOMENTS, nhwc_moments_kernel<T, V>, np.stat.grid, stream,
+                                              in<T>(data), set, np.stat.shape, partials, status)));
+    StatsSink sink{partials, np.stat.layout(), static_cast<float>(1.0 / pb.s), eps, mean, invstd};
+    launch(BNS_KERNEL_FINALIZE_STATS, finalize_stats_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, 1);
+    BNS_NHWC_BY_TYPE_V(pb.dtype, pb.C,
+                       (launch_grid(BNS_KERNEL_NORMALIZE, nhwc_normalize_kernel<T, V>, np.main.grid, stream, in<T>(x),
+                                    out<T>(y), gamma, beta, mean, invstd, static_cast<int>(np.rows), np.main.shape)));
+    if (virt && sp->yv)
+        BNS_NHWC_BY_TYPE_V(sp->xv_dtype, pb.C,
+                           (launch_grid(BNS_KERNEL_NORMALIZE, nhwc_normalize_kernel<T, V>, np.virt.grid, stream,
+                                        in<T>(sp->xv), out<T>(sp->yv), gamma, beta, mean, invstd,
+                                        static_cast<int>(np.sampled_rows), np.virt.shape)));
+    return last_error();
+}
+
+bns_status backward_nhwc_impl(const NhwcProblem& np, const bns_sampling* sp, const void* x, const void* dy,
+                              const float* gamma, const float* mean, const float* invstd, void* dx, float* dgamma,
+                              float* dbeta, void* ws, cudaStream_t stream) {
+    const Problem& pb = np.pb;
+    const bool full = pb.rule == BNS_RULE_FULL;
+    const bool virt = pb.rule == BNS_RULE_VIRTUAL;
+    float2* partials = ws_at<float2>(ws, np.off_bwd);
+    float2* partials_v = (virt && sp->dyv) ? ws_at<float2>(ws, np.off_bwd_v) : nullptr;
+    const int rows = static_cast<int>(np.rows);
+    if (full)
+        BNS_NHWC_BY_TYPE_V(pb.dtype, pb.C,
+                           (launch_grid(BNS_KERNEL_BWD_REDUCE, nhwc_bwd_reduce_kernel<T, V, false>, np.main.grid, stream,
+                                        in<T>(x), in<T>(dy), out<T>(nullptr), gamma, mean, invstd, rows, np.main.shape,
+                                        partials)));
+    else
+        BNS_NHWC_BY_TYPE_V(pb.dtype, pb.C,
+                           (launch_grid(BNS_KERNEL_BWD_REDUCE, nhwc_bwd_reduce_kernel<T, V, true>, np.main.grid, stream,
+                                        in<T>(x), in<T>(dy), out<T>(dx), gamma, mean, invstd, rows, np.main.shape,
+                                        partials)));
+    if (partials_v)
+        BNS_NHWC_BY_TYPE_V(sp->xv_dtype, pb.C,
+                           (launch_grid(BNS_KERNEL_BWD_REDUCE, nhwc_bwd_reduce_kernel<T, V, false>, np.virt.grid, stream,
+                                        in<T>(sp->xv), in<T>(sp->dyv), out<T>(nullptr), gamma, mean, invstd,
+                                        static_cast<int>(np.sampled_rows), np.virt.shape, partials_v)));
+    GradSink sink{partials, np.main.layout(), partials_v, np.virt.layout(), invstd, dgamma, dbeta};
+    launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, 1);
+    unsigned* status;
+    bns_status st = clear_status(pb, ws, stream, &status);
+    if (st != BNS_OK) return st;
+    const int* list = nullptr;
+    st = nhwc_stage_list(np, sp, ws, stream, &list);
+    if (st != BNS_OK) return st;
+    const RowSet set = nhwc_row_set(np, list);
+    const float inv_s = static_cast<float>(1.0 / pb.s);
+    if (virt) {
+        if (sp->dxv)
+            BNS_NHWC_BY_TYPE_V(sp->xv_dtype, pb.C,
+                               (launch_grid(BNS_KERNEL_COL_FIXUP, nhwc_fixup_kernel<T, V>, np.stat.grid, stream,
+                                            in<T>(sp->xv), in<T>(sp->dyv), out<T>(sp->dxv), gamma, mean, invstd, dgamma,
+                                            dbeta, inv_s, set, np.stat.shape, status)));
+    } else {
+        BNS_NHWC_BY_TYPE_V(pb.dtype, pb.C,
+                           (launch_grid(BNS_KERNEL_COL_FIXUP, nhwc_fixup_kernel<T, V>, np.stat.grid, stream, in<T>(x),
+                                        in<T>(dy), out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, set,
+                                        np.stat.shape, status)));
+    }
+    return last_error();
+}
+
 bns_sampling full_rule() {
     bns_sampling sp;
     std::memset(&sp, 0, sizeof(sp));
@@ -1119,6 +1323,42 @@ bns_status bns_backward_relu(const bns_shape* shape, const void* x, const void* 
                               pb.P)));
     }
     return last_error();
+}
+
+// ---------------------------------------------------------------------------------------- channels-last (NHWC)
+size_t bns_workspace_bytes_nhwc(const bns_shape* shape, const bns_sampling* sampling) {
+    NhwcProblem np;
+    if (make_nhwc(shape, sampling, np) != BNS_OK) return 0;
+    return np.total;
+}
+
+bns_status bns_forward_nhwc(const bns_shape* shape, const void* x, const float* gamma, const float* beta, float eps,
+                            const bns_sampling* sampling, void* y, float* mean, float* invstd, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream) {
+    NhwcProblem np;
+    bns_status st = make_nhwc(shape, sampling, np);
+    if (st != BNS_OK) return st;
+    if (!x || !gamma || !beta || !y || !mean || !invstd) return BNS_ERR_NULL;
+    if (!(eps > 0.f)) return BNS_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(y)) return BNS_ERR_ALIGN;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) || workspace_bytes < np.total)
+        return BNS_ERR_WORKSPACE;
+    return forward_nhwc_impl(np, sampling, x, gamma, beta, eps, y, mean, invstd, workspace,
+                             static_cast<cudaStream_t>(cuda_stream));
+}
+
+bns_status bns_backward_nhwc(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
+                             const float* mean, const float* invstd, const bns_sampling* sampling, void* dx,
+                             float* dgamma, float* dbeta, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    NhwcProblem np;
+    bns_status st = make_nhwc(shape, sampling, np);
+    if (st != BNS_OK) return st;
+    if (!x || !dy || !gamma || !mean || !invstd || !dx || !dgamma || !dbeta) return BNS_ERR_NULL;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dx)) return BNS_ERR_ALIGN;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) || workspace_bytes < np.total)
+        return BNS_ERR_WORKSPACE;
+    return backward_nhwc_impl(np, sampling, x, dy, gamma, mean, invstd, dx, dgamma, dbeta, workspace,
+                              static_cast<cudaStream_t>(cuda_stream));
 }
 
 // ---------------------------------------------------------------------------------------- no-allocation forward

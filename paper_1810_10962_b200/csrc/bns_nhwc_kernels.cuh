@@ -1,0 +1,262 @@
+// Channels-last (NHWC) kernels of the BN-sampling library (sm_100a).
+//
+// The paper's own layout (Appendix A: B in R^{N x H x W x C}, statistics reduce dims 0,1,2).  A tensor is
+// R = N*H*W rows of C contiguous channel values.  A thread owns V consecutive channels (up to 16 bytes)
+// for the whole kernel and walks down rows; a block is CW channel-vectors wide and RL row-lanes deep, so
+// one step of a block reads RL consecutive rows - contiguous memory when the block is as wide as a row.
+// Per-channel sums stay in registers, are folded across the row-lanes through shared memory once per
+// block, and the per-block partials are combined by the same finalize kernels as in the NCHW path (their
+// layout is the NCHW one with one position per channel).  A sampled pixel is a whole contiguous
+// channel vector here, which is what makes Feature Sampling cheap in this layout.
+#pragma once
+
+#include "bns_kernels.cuh"
+
+namespace bns {
+
+// Which rows of the tensor a kernel visits, enumerated q = 0 .. total-1.
+struct RowSet {
+    enum { kAll = 0, kSamples = 1, kPatches = 2 };
+    int mode;
+    int total;          // rows in the set
+    const int* list;    // kSamples: sample indices (device) or NULL for begin .. begin+count-1
+    int begin, HW;      // kSamples: row q belongs to sample q / HW
+    PatchRule patch;    // kPatches: shared or per-sample location (never per map: a row spans all channels)
+    int H, W;
+    __device__ __forceinline__ int row(int q, unsigned* status) const {
+        if (mode == kAll) return q;
+        if (mode == kSamples) {
+            const int i = q / HW;
+            return (list ? list[i] : begin + i) * HW + (q - i * HW);
+        }
+        const int PP = patch.ph * patch.pw;
+        const int n = q / PP, e = q - n * PP;
+        const int r = e / patch.pw, col = e - r * patch.pw;
+        int oh, ow;
+        patch_origin(patch, n, 0, H, W, status, oh, ow);
+        return n * (H * W) + (oh + r) * W + ow + col;
+    }
+};
+
+// Block shape: CW channel-vectors wide, RL row-lanes deep; grid.y tiles the channel-vectors.
+struct NhwcShape {
+    int C, V_unused, CV, CW, RL;  // channels, -, vectors per row, vectors per block, row-lanes per block
+    int rows_per_block;           // rows of the set that one block (grid.x) visits; a multiple of RL
+};
+
+struct NhwcThread {
+    int cv, rl;    // channel-vector of the row, row-lane
+    bool active;
+    __device__ __forceinline__ NhwcThread(const NhwcShape& s) {
+        const int t = threadIdx.x;
+        const int cvi = t % s.CW;
+        rl = t / s.CW;
+        cv = blockIdx.y * s.CW + cvi;
+        active = rl < s.RL && cv < s.CV;
+    }
+};
+
+// ------------------------------------------------------------------------------------ statistics
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+nhwc_moments_kernel(const typename T::storage* __restrict__ x, RowSet set, NhwcShape s, float4* __restrict__ partials,
+                    unsigned* status) {
+    __shared__ float s_cnt[kThreads], s_mean[kThreads * V], s_m2[kThreads * V];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const NhwcThread me(s);
+    const int q0 = blockIdx.x * s.rows_per_block, q1 = min(set.total, q0 + s.rows_per_block);
+    float K[V], s1[V], s2[V], cnt = 0.f;
+#pragma unroll
+    for (int j = 0; j < V; ++j) K[j] = s1[j] = s2[j] = 0.f;
+    if (me.active) {
+        const typename T::storage* xp = x + static_cast<size_t>(me.cv) * V;
+        for (int q = q0 + me.rl; q < q1; q += kUnroll * s.RL) {
+            Vec<T, V> v[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                if (q + u * s.RL < q1) v[u].load(xp + static_cast<size_t>(set.row(q + u * s.RL, status)) * s.C);
+            if (cnt == 0.f) {
+#pragma unroll
+                for (int j = 0; j < V; ++j) K[j] = v[0].get(j);  // pivot: the thread's first row
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                if (q + u * s.RL < q1) {
+#pragma unroll
+                    for (int j = 0; j < V; ++j) {
+                        float d = v[u].get(j) - K[j];
+                        s1[j] += d;
+                        s2[j] = fmaf(d, d, s2[j]);
+                    }
+                    cnt += 1.f;
+                }
+        }
+    }
+    s_cnt[threadIdx.x] = cnt;
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        Moments m = from_shifted_sums(cnt, K[j], s1[j], s2[j]);
+        s_mean[threadIdx.x * V + j] = m.mean;
+        s_m2[threadIdx.x * V + j] = m.m2;
+    }
+    __syncthreads();
+    // channel ch of the block (ch < CW*V): merge its RL row-lane entries in lane order
+    for (int ch = threadIdx.x; ch < s.CW * V; ch += kThreads) {
+        const int cvi = ch / V, j = ch - cvi * V;
+        const int c = (blockIdx.y * s.CW + cvi) * V + j;
+        if (c >= s.C) continue;
+        Moments acc = {0.f, 0.f, 0.f};
+        for (int rl = 0; rl < s.RL; ++rl) {
+            const int t = rl * s.CW + cvi;
+            acc = merge(acc, Moments{s_cnt[t], s_mean[t * V + j], s_m2[t * V + j]});
+        }
+        partials[static_cast<size_t>(blockIdx.x) * s.C + c] = make_float4(acc.cnt, acc.mean, acc.m2, 0.f);
+    }
+}
+
+// ------------------------------------------------------------------------------------ normalise + affine
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+nhwc_normalize_kernel(const typename T::storage* __restrict__ x, typename T::storage* __restrict__ y,
+                      const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
+                      const float* __restrict__ invstd, int rows, NhwcShape s) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const NhwcThread me(s);
+    if (!me.active) return;
+    float a[V], b[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        const int c = me.cv * V + j;
+        a[j] = gamma[c] * invstd[c];
+        b[j] = fmaf(-mean[c], a[j], beta[c]);
+    }
+    const int q0 = blockIdx.x * s.rows_per_block, q1 = min(rows, q0 + s.rows_per_block);
+    const size_t col = static_cast<size_t>(me.cv) * V;
+    for (int q = q0 + me.rl; q < q1; q += kUnroll * s.RL) {
+        Vec<T, V> v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (q + u * s.RL < q1) v[u].load(x + static_cast<size_t>(q + u * s.RL) * s.C + col);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (q + u * s.RL < q1) {
+#pragma unroll
+                for (int j = 0; j < V; ++j) v[u].set(j, fmaf(a[j], v[u].get(j), b[j]));
+                v[u].store(y + static_cast<size_t>(q + u * s.RL) * s.C + col);
+            }
+    }
+}
+
+// ------------------------------------------------------------------------------------ backward, pass 1
+template <typename T, int V, bool WRITE_DX>
+__global__ void __launch_bounds__(kThreads)
+nhwc_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
+                       typename T::storage* __restrict__ dx, const float* __restrict__ gamma,
+                       const float* __restrict__ mean, const float* __restrict__ invstd, int rows, NhwcShape s,
+                       float2* __restrict__ partials) {
+    __shared__ float s_dy[kThreads * V], s_dyxc[kThreads * V];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const NhwcThread me(s);
+    float acc_dy[V], acc_dyxc[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc_dy[j] = acc_dyxc[j] = 0.f;
+    if (me.active) {
+        float a[V], mu[V];
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            const int c = me.cv * V + j;
+            mu[j] = mean[c];
+            a[j] = WRITE_DX ? gamma[c] * invstd[c] : 0.f;
+        }
+        const int q0 = blockIdx.x * s.rows_per_block, q1 = min(rows, q0 + s.rows_per_block);
+        const size_t col = static_cast<size_t>(me.cv) * V;
+        for (int q = q0 + me.rl; q < q1; q += kUnroll * s.RL) {
+            Vec<T, V> vx[kUnroll], vg[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                if (q + u * s.RL < q1) {
+                    const size_t off = static_cast<size_t>(q + u * s.RL) * s.C + col;
+                    vx[u].load(x + off);
+                    vg[u].load(dy + off);
+                }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                if (q + u * s.RL < q1) {
+#pragma unroll
+                    for (int j = 0; j < V; ++j) {
+                        float g = vg[u].get(j);
+                        acc_dy[j] += g;
+                        acc_dyxc[j] = fmaf(g, vx[u].get(j) - mu[j], acc_dyxc[j]);
+                        if (WRITE_DX) vg[u].set(j, a[j] * g);
+                    }
+                    if (WRITE_DX) vg[u].store(dx + static_cast<size_t>(q + u * s.RL) * s.C + col);
+                }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        s_dy[threadIdx.x * V + j] = acc_dy[j];
+        s_dyxc[threadIdx.x * V + j] = acc_dyxc[j];
+    }
+    __syncthreads();
+    for (int ch = threadIdx.x; ch < s.CW * V; ch += kThreads) {
+        const int cvi = ch / V, j = ch - cvi * V;
+        const int c = (blockIdx.y * s.CW + cvi) * V + j;
+        if (c >= s.C) continue;
+        float sa = 0.f, sb = 0.f;
+        for (int rl = 0; rl < s.RL; ++rl) {
+            const int t = rl * s.CW + cvi;
+            sa += s_dy[t * V + j];
+            sb += s_dyxc[t * V + j];
+        }
+        partials[static_cast<size_t>(blockIdx.x) * s.C + c] = make_float2(sa, sb);
+    }
+}
+
+// ------------------------------------------------------------------------------------ backward, statistics terms
+// dx = a dy - A - Q (x - mean) on the rows of the set; dy == NULL reads as zeros.
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+nhwc_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
+                  typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
+                  const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
+                  float inv_s, RowSet set, NhwcShape s, unsigned* status) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const NhwcThread me(s);
+    if (!me.active) return;
+    FixCoef k[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        const int c = me.cv * V + j;
+        k[j] = fix_coef(gamma[c], mean[c], invstd[c], dgamma[c], dbeta[c], inv_s);
+    }
+    const int q0 = blockIdx.x * s.rows_per_block, q1 = min(set.total, q0 + s.rows_per_block);
+    const size_t col = static_cast<size_t>(me.cv) * V;
+    for (int q = q0 + me.rl; q < q1; q += kUnroll * s.RL) {
+        Vec<T, V> vx[kUnroll], vg[kUnroll];
+        size_t off[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (q + u * s.RL < q1) {
+                off[u] = static_cast<size_t>(set.row(q + u * s.RL, status)) * s.C + col;
+                vx[u].load(x + off[u]);
+                if (dy) vg[u].load(dy + off[u]);
+            }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (q + u * s.RL < q1) {
+#pragma unroll
+                for (int j = 0; j < V; ++j) {
+                    float g = dy ? vg[u].get(j) : 0.f;
+                    vg[u].set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (vx[u].get(j) - k[j].mu));
+                }
+                vg[u].store(dx + off[u]);
+            }
+    }
+}
+
+}  // namespace bns

@@ -183,3 +183,75 @@ def test_fused_residual_relu(rule, kw, dtype, dims, with_residual):
         assert np.array_equal(_to_host(dres), dres_want.astype(np.float32))     # dy or 0: bit-exact
     else:
         assert dres is None
+
+
+def _nhwc(a):
+    return np.ascontiguousarray(np.transpose(a, (0, 2, 3, 1)))
+
+
+def _nchw(a):
+    return np.ascontiguousarray(np.transpose(a, (0, 3, 1, 2)))
+
+
+NHWC_CASES = [
+    ("batch", dict(k=5, contiguous=False)), ("batch", dict(k=3)), ("feature", dict(ph=3, pw=4, offset_mode=0)),
+    ("feature", dict(ph=2, pw=2, offset_mode=1)), ("feature", dict(ph=1, pw=1, offset_mode=0)),
+    ("virtual", dict(nv=2)), ("virtual", dict(nv=1, with_dyv=False)), ("full", dict()),
+]
+
+
+@pytest.mark.parametrize("rule,kw", NHWC_CASES)
+@pytest.mark.parametrize("dtype,dims", [("f32", (12, 64, 9, 11)), ("bf16", (10, 40, 7, 7)), ("f32", (6, 7, 5, 3)),
+                                        ("bf16", (3, 2080, 2, 2)), ("f32", (40, 16, 16, 16))])
+def test_channels_last_layout(rule, kw, dtype, dims):
+    """The NHWC entry points against the (NCHW) oracle on the transposed tensors."""
+    import torch
+    from paper_1810_10962_b200 import bns
+    kw = dict(kw)
+    N, C, H, W = dims
+    if rule == "batch":
+        kw["k"] = min(kw["k"], N)
+    if rule == "feature":
+        kw["ph"], kw["pw"] = min(kw["ph"], H), min(kw["pw"], W)
+    if rule == "virtual":
+        kw["xv_dtype"] = dtype
+    case = make_case(N, C, H, W, rule, seed=97, dtype=dtype, **kw)
+    dev = lambda a, d=dtype: _to_device(_nhwc(a), d)
+    x, dy = dev(case.x), dev(case.dy)
+    gamma, beta = torch.from_numpy(case.gamma).cuda(), torch.from_numpy(case.beta).cuda()
+    if rule == "full":
+        sp = bns.Sampling.full()
+    elif rule == "batch":
+        sp = bns.Sampling.batch(case.sample_idx)
+    elif rule == "feature":
+        off = case.offsets if case.offset_mode == 0 else torch.from_numpy(case.offsets).cuda()
+        sp = bns.Sampling.feature(case.ph, case.pw, off, case.offset_mode)
+    else:
+        xv = dev(case.xv, case.xv_dtype)
+        dyv = None if case.dyv is None else dev(case.dyv, case.xv_dtype)
+        sp = bns.Sampling.virtual(xv, yv=torch.empty_like(xv), dyv=dyv, dxv=torch.empty_like(xv))
+    y, mean, invstd, ws = bns.forward_nhwc(x, gamma, beta, case.eps, sp)
+    dx, dgamma, dbeta = bns.backward_nhwc(x, dy, gamma, mean, invstd, sp, ws)
+    torch.cuda.synchronize()
+    from helpers import run_oracle
+    f, b = run_oracle(case)
+    tensor_close = close_f32 if dtype == "f32" else close_bf16
+    close_f32(mean.cpu().numpy(), f.mean, "mean")
+    close_f32(invstd.cpu().numpy(), f.invstd, "invstd")
+    tensor_close(_nchw(_to_host(y)), f.y, "y")
+    tensor_close(_nchw(_to_host(dx)), b.dx, "dx")
+    close_f32(dgamma.cpu().numpy(), b.dgamma, "dgamma")
+    close_f32(dbeta.cpu().numpy(), b.dbeta, "dbeta")
+    if rule == "virtual":
+        tensor_close(_nchw(_to_host(sp.yv)), f.yv, "yv")
+        tensor_close(_nchw(_to_host(sp.dxv)), b.dxv, "dxv")
+
+
+def test_channels_last_rejects_per_map_offsets():
+    import torch
+    from paper_1810_10962_b200 import bns
+    x = torch.zeros(2, 4, 4, 8, device="cuda")
+    off = torch.zeros(2 * 8, 2, dtype=torch.int32, device="cuda")
+    g = torch.ones(8, device="cuda")
+    with pytest.raises(bns.BnsError):
+        bns.forward_nhwc(x, g, g, 1e-5, bns.Sampling.feature(2, 2, off, bns.OFF_PER_MAP))
