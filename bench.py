@@ -226,15 +226,17 @@ def measured_hbm_peak():
 class DeviceLayer:
     """Device buffers of one layer (several rotating sets of x, dy, y, dx) and its launch closures."""
 
-    def __init__(self, layer: Layer, host, sets, torch, bns, full_bn=False):
+    def __init__(self, layer: Layer, host, sets, torch, bns, full_bn=False, nhwc=False):
         self.layer, self.bns, self.torch = layer, bns, torch
         self.full = full_bn or layer.rule == "full"
         self.mixed = layer.rule == "mixed" and not self.full
         self.relu = layer.rule == "relu"      # the full-BN comparison runs through the same fused kernels
+        self.nhwc = nhwc
         dt = torch.float32 if layer.dtype == "f32" else torch.bfloat16
 
         def dev(a):
-            return torch.from_numpy(a).cuda().to(dt)        # exact: the values are representable in dt
+            t = torch.from_numpy(a).cuda().to(dt)           # exact: the values are representable in dt
+            return t.permute(0, 2, 3, 1).contiguous() if nhwc else t
 
         x, dy = dev(host["x"]), dev(host["dy"])
         self.sets = [(x, dy, torch.empty_like(x), torch.empty_like(x))]
@@ -243,6 +245,17 @@ class DeviceLayer:
         self.gamma, self.beta = torch.from_numpy(host["gamma"]).cuda(), torch.from_numpy(host["beta"]).cuda()
         C = layer.C
         self.mean, self.invstd, self.dgamma, self.dbeta = (torch.empty(C, device="cuda") for _ in range(4))
+        if nhwc:
+            if layer.rule not in ("batch", "feature", "full"):
+                raise SystemExit("--layout nhwc is benchmarked for the batch, feature and full rules")
+            if self.full:
+                self.sp = bns.Sampling.full()
+            elif layer.rule == "batch":
+                self.sp = bns.Sampling.batch(host["sample_idx"])
+            else:
+                self.sp = bns.Sampling.feature(layer.kw["ph"], layer.kw["pw"], host["offsets"])
+            self.ws = None
+            return
         if self.relu:
             self.sp = (bns.Sampling.full() if self.full
                        else bns.Sampling.feature(layer.kw["ph"], layer.kw["pw"], host["offsets"]))
@@ -272,6 +285,12 @@ class DeviceLayer:
                       for sx, sdy, sy, sdx in self.sets]
 
     def step(self, i):
+        if self.nhwc:
+            x, dy, _, _ = self.sets[i % len(self.sets)]
+            b = self.bns
+            _, mean, invstd, self.ws = b.forward_nhwc(x, self.gamma, self.beta, EPS, self.sp, workspace=self.ws)
+            b.backward_nhwc(x, dy, self.gamma, mean, invstd, self.sp, self.ws)
+            return
         if self.relu:
             x, dy, _, _ = self.sets[i % len(self.sets)]
             b = self.bns
@@ -406,8 +425,10 @@ def run_ours(args):
     bytes_per_tensor_set = sum(4 * l.elems * l.ebytes for l in layers)
     # rotate buffer sets so that no tensor is reused before > 2x L2 (126 MB) of other data went by
     sets = 2 if bytes_per_tensor_set >= 512e6 else min(8, max(2, int(np.ceil(512e6 / bytes_per_tensor_set))))
-    dev = [DeviceLayer(l, h, sets, torch, bns) for l, h in zip(layers, hosts)]
-    full = [DeviceLayer(l, h, sets, torch, bns, full_bn=True) for l, h in zip(layers, hosts)] if args.full_bn else []
+    nhwc = args.layout == "nhwc"
+    dev = [DeviceLayer(l, h, sets, torch, bns, nhwc=nhwc) for l, h in zip(layers, hosts)]
+    full = ([DeviceLayer(l, h, sets, torch, bns, full_bn=True, nhwc=nhwc) for l, h in zip(layers, hosts)]
+            if args.full_bn else [])
 
     def step(i):
         for d in dev:
@@ -470,7 +491,7 @@ def run_ours(args):
         # from the vectors the two forward calls above left behind (diagnostic; synthetic activations)
         torch.cuda.synchronize()
         for d, f in zip(dev, full):
-            if d.relu:
+            if d.relu or d.nhwc:
                 continue                      # that path keeps its statistics in tensors of its own
             sigma_s, sigma = 1.0 / d.invstd.double(), 1.0 / f.invstd.double()     # sqrt(var + eps) each
             per_layer[d.layer.name]["estimation_error"] = {
@@ -492,7 +513,7 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     e2e = None
-    if args.e2e and rank == 0:
+    if args.e2e and rank == 0 and not nhwc:
         e2e = run_e2e(torch, bns, layers, hosts, max(2, min(args.steps, args.e2e_steps)))
     if world > 1:
         dist.barrier()
@@ -510,7 +531,7 @@ def run_ours(args):
             "config": {"workload": args.workload + (f" (only {args.only})" if args.only else ""),
                        "layers": [f"{l.name}:{l.N}x{l.C}x{l.H}x{l.W}:{l.dtype}:x{l.count}" for l in layers],
                        "step": "forward+backward of every layer", "algorithmic_bytes_per_step": step_bytes,
-                       "cache": f"inputs larger than L2; {sets} buffer sets rotated", "replicas": world,
+                       "cache": f"inputs larger than L2; {sets} buffer sets rotated", "replicas": world, "layout": args.layout,
                        "launch": f"CUDA graph replay, {sets} steps per graph" if graphed else "eager launches",
                        "tuning": args.tune},
             "frac_of_hbm_peak": round(value / world / peak, 4), "hbm_peak_gbs": peak, "hbm_peak_source": peak_source,
@@ -675,6 +696,8 @@ def main():
     ap.add_argument("--tune", action="append", default=[], metavar="NAME=VALUE",
                     help="launch-shape knob of the library (bns_set_tuning), e.g. --tune pdl=0")
     ap.add_argument("--no-full-bn", dest="full_bn", action="store_false", help="skip the full-BN comparison")
+    ap.add_argument("--layout", choices=["nchw", "nhwc"], default="nchw",
+                    help="tensor layout of the timed calls (nhwc: the channels-last entry points)")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="time eager launches instead of replaying a CUDA graph of the step")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false", help="skip the host-buffer end-to-end leg")

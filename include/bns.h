@@ -336,7 +336,8 @@ const char* bns_kernel_name(int kernel_kind);
  * per block of the streaming kernels; "stat_target_blocks" / "stat_min_chunk": the same for the
  * statistics kernels; "direct_max": sampled elements per channel up to which one block per channel computes the
  * statistics (and, in the backward, combines the sums and applies the statistics terms) without
- * partial sums, 0 = never; "pdl": 0/1 programmatic dependent launch; "l2_order": 0/1 visit rows in an
+ * partial sums, 0 = never; "nhwc_blocks": blocks per launch of the channels-last kernels (each block leaves one partial per
+ * channel); "pdl": 0/1 programmatic dependent launch; "l2_order": 0/1 visit rows in an
  * order that lets a kernel find in L2 what the previous one read.  Returns BNS_OK,
  * BNS_ERR_RULE for an unknown name or BNS_ERR_SHAPE for a value < 1. */
 int bns_set_tuning(const char* name, int value);

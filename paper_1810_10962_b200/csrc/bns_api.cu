@@ -648,13 +648,12 @@ bns_status backward_mixed_impl(const MixedProblem& mp, const bns_sampling* sp, c
 }
 
 // ------------------------------------------------------------------------------------ channels-last (NHWC)
+int g_nhwc_blocks = kSmCount * 8;  // blocks per channels-last launch
+
 struct NhwcLaunch {
     NhwcShape shape;
     dim3 grid;
     size_t partial_count() const { return static_cast<size_t>(grid.x) * shape.C; }
-    PartialLayout layout() const {  // the NCHW layout with one position per channel and a single tile
-        return PartialLayout{static_cast<int>(grid.x), 1u, 0x7fffffffu, shape.C};
-    }
 };
 
 // Block shape and grid for visiting `total` rows of C channels.
@@ -669,7 +668,10 @@ NhwcLaunch plan_nhwc(int C, int ebytes, long total, bool statistics) {
     s.CW = std::min(s.CV, kThreads);
     s.RL = kThreads / s.CW;
     const int gy = (s.CV + s.CW - 1) / s.CW;
-    const long target = std::max(1L, static_cast<long>(statistics ? g_stat_target_blocks : g_target_blocks) / gy);
+    // few, long-lived blocks: every block leaves one partial per channel, so the block count is also the
+    // number of partials the finalize kernels have to read per channel
+    (void)statistics;
+    const long target = std::max(1L, static_cast<long>(g_nhwc_blocks) / gy);
     long rpb = std::max<long>(static_cast<long>(s.RL) * kUnroll * 2, (total + target - 1) / target);
     rpb = (rpb + s.RL - 1) / s.RL * s.RL;
     s.rows_per_block = static_cast<int>(rpb);
@@ -757,11 +759,11 @@ bns_status nhwc_stage_list(const NhwcProblem& np, const bns_sampling* sp, void* 
     } while (0)
 
 template <typename... KArgs, typename... Args>
-void launch_grid(int kind, void (*kernel)(KArgs...), dim3 grid, cudaStream_t s, Args&&... args) {
+void launch_grid_block(int kind, void (*kernel)(KArgs...), dim3 grid, int threads, cudaStream_t s, Args&&... args) {
     LaunchScope scope(kind, s);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(threads);
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -769,6 +771,11 @@ void launch_grid(int kind, void (*kernel)(KArgs...), dim3 grid, cudaStream_t s, 
     cfg.attrs = attr;
     cfg.numAttrs = g_pdl ? 1 : 0;
     cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+template <typename... KArgs, typename... Args>
+void launch_grid(int kind, void (*kernel)(KArgs...), dim3 grid, cudaStream_t s, Args&&... args) {
+    launch_grid_block(kind, kernel, grid, kThreads, s, static_cast<Args&&>(args)...);
 }
 
 bns_status forward_nhwc_impl(const NhwcProblem& np, const bns_sampling* sp, const void* x, const float* gamma,
@@ -788,8 +795,9 @@ bns_status forward_nhwc_impl(const NhwcProblem& np, const bns_sampling* sp, cons
     float4* partials = ws_at<float4>(ws, np.off_stats);
     BNS_NHWC_BY_TYPE_V(dt, pb.C, (launch_grid(BNS_KERNEL_COL_MOMENTS, nhwc_moments_kernel<T, V>, np.stat.grid, stream,
                                               in<T>(data), set, np.stat.shape, partials, status)));
-    StatsSink sink{partials, np.stat.layout(), static_cast<float>(1.0 / pb.s), eps, mean, invstd};
-    launch(BNS_KERNEL_FINALIZE_STATS, finalize_stats_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, 1);
+    launch_grid_block(BNS_KERNEL_FINALIZE_STATS, nhwc_finalize_stats_kernel, dim3((pb.C + 31) / 32), kFinalizeThreads,
+                      stream, static_cast<const float4*>(partials), static_cast<int>(np.stat.grid.x), pb.C, static_cast<float>(1.0 / pb.s),
+           eps, mean, invstd);
     BNS_NHWC_BY_TYPE_V(pb.dtype, pb.C,
                        (launch_grid(BNS_KERNEL_NORMALIZE, nhwc_normalize_kernel<T, V>, np.main.grid, stream, in<T>(x),
                                     out<T>(y), gamma, beta, mean, invstd, static_cast<int>(np.rows), np.main.shape)));
@@ -825,8 +833,9 @@ bns_status backward_nhwc_impl(const NhwcProblem& np, const bns_sampling* sp, con
                            (launch_grid(BNS_KERNEL_BWD_REDUCE, nhwc_bwd_reduce_kernel<T, V, false>, np.virt.grid, stream,
                                         in<T>(sp->xv), in<T>(sp->dyv), out<T>(nullptr), gamma, mean, invstd,
                                         static_cast<int>(np.sampled_rows), np.virt.shape, partials_v)));
-    GradSink sink{partials, np.main.layout(), partials_v, np.virt.layout(), invstd, dgamma, dbeta};
-    launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, 1);
+    launch_grid_block(BNS_KERNEL_FINALIZE_BWD, nhwc_finalize_bwd_kernel, dim3((pb.C + 31) / 32), kFinalizeThreads, stream,
+                      static_cast<const float2*>(partials), static_cast<int>(np.main.grid.x),
+           static_cast<const float2*>(partials_v), static_cast<int>(np.virt.grid.x), pb.C, invstd, dgamma, dbeta);
     unsigned* status;
     bns_status st = clear_status(pb, ws, stream, &status);
     if (st != BNS_OK) return st;
@@ -1037,7 +1046,7 @@ int bns_set_tuning(const char* name, int value) {
         bool* bvalue;
     } knobs[] = {{"target_blocks", &g_target_blocks, nullptr},   {"min_chunk", &g_min_chunk, nullptr},
                  {"stat_target_blocks", &g_stat_target_blocks, nullptr}, {"stat_min_chunk", &g_stat_min_chunk, nullptr},
-                 {"direct_max", &g_direct_max, nullptr},         {"pdl", nullptr, &g_pdl},                       {"l2_order", nullptr, &g_l2_order}};
+                 {"direct_max", &g_direct_max, nullptr},         {"nhwc_blocks", &g_nhwc_blocks, nullptr},         {"pdl", nullptr, &g_pdl},                       {"l2_order", nullptr, &g_l2_order}};
     for (const Knob& k : knobs) {
         if (std::strcmp(name, k.name) != 0) continue;
         if (k.ivalue) {

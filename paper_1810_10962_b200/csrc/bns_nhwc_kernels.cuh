@@ -5,9 +5,9 @@
 // for the whole kernel and walks down rows; a block is CW channel-vectors wide and RL row-lanes deep, so
 // one step of a block reads RL consecutive rows - contiguous memory when the block is as wide as a row.
 // Per-channel sums stay in registers, are folded across the row-lanes through shared memory once per
-// block, and the per-block partials are combined by the same finalize kernels as in the NCHW path (their
-// layout is the NCHW one with one position per channel).  A sampled pixel is a whole contiguous
-// channel vector here, which is what makes Feature Sampling cheap in this layout.
+// block, and the per-block partials (one per channel and block) are combined in a fixed order by the
+// finalize kernels at the end of this file.  A sampled pixel is a whole contiguous channel vector here,
+// which is what makes Feature Sampling cheap in this layout.
 #pragma once
 
 #include "bns_kernels.cuh"
@@ -256,6 +256,92 @@ nhwc_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::s
                 }
                 vg[u].store(dx + off[u]);
             }
+    }
+}
+
+// ------------------------------------------------------------------------------------ combining the blocks' partials
+// Every block of a channels-last pass leaves one partial per channel: partial[block*C + c].  Here lane l
+// of a warp owns channel 32*blockIdx.x + l (neighbouring lanes read neighbouring addresses) and the 32
+// warps of a 1024-thread block share the entries, each loading a batch before it adds; the warps' results
+// meet in shared memory and are combined in warp order.
+constexpr int kFinalizeThreads = 1024;
+constexpr int kFinalizeWarps = kFinalizeThreads / 32;
+
+__global__ void __launch_bounds__(kFinalizeThreads)
+nhwc_finalize_stats_kernel(const float4* __restrict__ partials, int entries, int C, float inv_s, float eps,
+                           float* __restrict__ mean, float* __restrict__ invstd) {
+    __shared__ float s_cnt[kFinalizeThreads], s_mean[kFinalizeThreads], s_m2[kFinalizeThreads];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int c = blockIdx.x * 32 + lane;
+    Moments acc = {0.f, 0.f, 0.f};
+    if (c < C) {
+        constexpr int kBatch = 4;
+        for (int e = warp; e < entries; e += kBatch * kFinalizeWarps) {
+            float4 v[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u)
+                v[u] = e + u * kFinalizeWarps < entries ? partials[static_cast<size_t>(e + u * kFinalizeWarps) * C + c]
+                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) acc = merge(acc, Moments{v[u].x, v[u].y, v[u].z});
+        }
+    }
+    s_cnt[threadIdx.x] = acc.cnt;
+    s_mean[threadIdx.x] = acc.mean;
+    s_m2[threadIdx.x] = acc.m2;
+    __syncthreads();
+    if (warp == 0 && c < C) {
+        Moments tot = {0.f, 0.f, 0.f};
+        for (int w = 0; w < kFinalizeWarps; ++w)
+            tot = merge(tot, Moments{s_cnt[w * 32 + lane], s_mean[w * 32 + lane], s_m2[w * 32 + lane]});
+        mean[c] = tot.mean;
+        invstd[c] = 1.0f / sqrtf(tot.m2 * inv_s + eps);
+    }
+}
+
+__global__ void __launch_bounds__(kFinalizeThreads)
+nhwc_finalize_bwd_kernel(const float2* __restrict__ partials, int entries, const float2* __restrict__ partials_v,
+                         int entries_v, int C, const float* __restrict__ invstd, float* __restrict__ dgamma,
+                         float* __restrict__ dbeta) {
+    __shared__ float s_a[kFinalizeThreads], s_b[kFinalizeThreads];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int c = blockIdx.x * 32 + lane;
+    float sa = 0.f, sb = 0.f;
+    if (c < C) {
+        constexpr int kBatch = 4;
+        for (int pass = 0; pass < 2; ++pass) {
+            const float2* src = pass ? partials_v : partials;
+            const int n = pass ? entries_v : entries;
+            if (!src) continue;
+            for (int e = warp; e < n; e += kBatch * kFinalizeWarps) {
+                float2 v[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u)
+                    v[u] = e + u * kFinalizeWarps < n ? src[static_cast<size_t>(e + u * kFinalizeWarps) * C + c]
+                                                      : make_float2(0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    sa += v[u].x;
+                    sb += v[u].y;
+                }
+            }
+        }
+    }
+    s_a[threadIdx.x] = sa;
+    s_b[threadIdx.x] = sb;
+    __syncthreads();
+    if (warp == 0 && c < C) {
+        float ta = 0.f, tb = 0.f;
+        for (int w = 0; w < kFinalizeWarps; ++w) {
+            ta += s_a[w * 32 + lane];
+            tb += s_b[w * 32 + lane];
+        }
+        dbeta[c] = ta;
+        dgamma[c] = tb * invstd[c];
     }
 }
 
