@@ -282,7 +282,10 @@ bns_status bns_forward_static(const bns_shape* shape, const void* x, const float
  * x, dy, y, dx, gamma, beta and the six outputs are HOST pointers (pinned memory lets the copies
  * run asynchronously); pointers inside `sampling` keep the meaning documented above.
  * `arena` is DEVICE scratch of at least bns_host_arena_bytes() bytes, 256-byte aligned.
- * Everything is enqueued on `cuda_stream`; synchronise it before reading the outputs.
+ * Everything is enqueued on `cuda_stream` (the copy of y runs on a helper stream of the library so
+ * that it overlaps the upload of dy, and joins `cuda_stream` again before the call's last copies);
+ * synchronise `cuda_stream` before reading the outputs.  The helper stream and two events are created
+ * on the first call on a device and kept: the one exception to "keeps no state".
  * The paper has no counterpart (its measurements include input pipelines only as a whole).
  */
 size_t bns_host_arena_bytes(const bns_shape* shape, const bns_sampling* sampling);

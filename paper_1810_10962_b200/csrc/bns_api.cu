@@ -868,6 +868,33 @@ bns_sampling full_rule() {
 
 }  // namespace
 
+// Helper stream and events of bns_forward_backward_host, one set per device, created on first use and
+// kept until the process ends (the only objects this library ever creates).  NULL if creation fails: the
+// call then runs on the caller's stream alone.
+struct CopyLane {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t forward_done = nullptr, y_done = nullptr;
+    bool tried = false;
+};
+CopyLane g_copy_lanes[64];
+
+CopyLane* copy_lane() {
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return nullptr;
+    CopyLane& lane = g_copy_lanes[device];
+    if (!lane.tried) {
+        lane.tried = true;
+        bool ok = cudaStreamCreateWithFlags(&lane.stream, cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&lane.forward_done, cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&lane.y_done, cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
+            cudaGetLastError();
+            lane.stream = nullptr;
+        }
+    }
+    return lane.stream ? &lane : nullptr;
+}
+
 // ======================================================================================== C ABI
 extern "C" {
 
@@ -953,11 +980,22 @@ bns_status bns_forward_backward_host(const bns_shape* shape, const void* x, cons
     if (!ok) return BNS_ERR_CUDA;
     st = forward_impl(pb, sampling, d_x, d_gamma, d_beta, eps, d_y, d_mean, d_invstd, ws, stream);
     if (st != BNS_OK) return st;
-    ok &= cudaMemcpyAsync(y, d_y, tbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    // y travels to the host on a helper stream while dy travels to the device on the caller's: the two
+    // directions of the link are independent.  The helper joins the caller's stream again at the end.
+    CopyLane* lane = copy_lane();
+    if (lane) {
+        ok &= cudaEventRecord(lane->forward_done, stream) == cudaSuccess;
+        ok &= cudaStreamWaitEvent(lane->stream, lane->forward_done, 0) == cudaSuccess;
+        ok &= cudaMemcpyAsync(y, d_y, tbytes, cudaMemcpyDeviceToHost, lane->stream) == cudaSuccess;
+        ok &= cudaEventRecord(lane->y_done, lane->stream) == cudaSuccess;
+    } else {
+        ok &= cudaMemcpyAsync(y, d_y, tbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    }
     ok &= cudaMemcpyAsync(d_dy, dy, tbytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
     if (!ok) return BNS_ERR_CUDA;
     st = backward_impl(pb, sampling, d_x, d_dy, d_gamma, d_mean, d_invstd, d_dx, d_dgamma, d_dbeta, ws, stream);
     if (st != BNS_OK) return st;
+    if (lane) ok &= cudaStreamWaitEvent(stream, lane->y_done, 0) == cudaSuccess;
     ok &= cudaMemcpyAsync(dx, d_dx, tbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     ok &= cudaMemcpyAsync(mean, d_mean, vbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     ok &= cudaMemcpyAsync(invstd, d_invstd, vbytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
