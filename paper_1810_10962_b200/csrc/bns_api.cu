@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "bns_kernels.cuh"
@@ -877,10 +878,12 @@ struct CopyLane {
     bool tried = false;
 };
 CopyLane g_copy_lanes[64];
+std::mutex g_copy_lanes_mutex;
 
 CopyLane* copy_lane() {
     int device = -1;
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return nullptr;
+    std::lock_guard<std::mutex> guard(g_copy_lanes_mutex);
     CopyLane& lane = g_copy_lanes[device];
     if (!lane.tried) {
         lane.tried = true;
