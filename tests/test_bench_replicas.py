@@ -90,3 +90,28 @@ def test_shared_statistics_exchange_between_two_ranks():
         assert gathered == [[[1.0] * 4] * 3, [[2.0] * 4] * 3]       # rank-major, same on every rank
         assert sums == [[3.0] * 4] * 2
         assert rows == [[float(rank + 1)] * 4] * 3                  # the input is left alone
+
+
+def test_reference_arm_prints_one_json_line_with_the_agreed_keys():
+    """`bench.py --impl reference` times the CPU oracle; it needs no GPU, so its output format is checked here."""
+    import json
+    import subprocess
+    run = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                          "--steps", "2", "--warmup", "1"], capture_output=True, text=True, cwd=ROOT, timeout=300)
+    assert run.returncode == 0, run.stderr
+    lines = [l for l in run.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["unit"] == "GB/s" and d["higher_is_better"] is True
+    assert d["metric"] == "sampled_bn_fwd_bwd_algorithmic_gbps" and d["value"] > 0 and d["steps"] == 2
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
+    assert d["e2e"] == {"value": d["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    assert d["config"]["workload"] == "tiny" and d["vs_baseline"] is None
+
+
+def test_other_ranks_of_the_reference_arm_stay_silent():
+    import subprocess
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    run = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                          "--gpus", "2"], capture_output=True, text=True, cwd=ROOT, env=env, timeout=300)
+    assert run.returncode == 0 and run.stdout.strip() == ""
