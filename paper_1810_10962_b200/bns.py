@@ -238,6 +238,19 @@ def _dev(t: torch.Tensor) -> int:
     return t.data_ptr()
 
 
+def _like(t: torch.Tensor, x: torch.Tensor, name: str) -> int:
+    """Device pointer of a tensor that must match x in shape and element type (outputs are written in full)."""
+    if t.shape != x.shape or t.dtype != x.dtype:
+        raise TypeError(f"{name} must have the shape and dtype of x")
+    return _dev(t)
+
+
+def _check_virtual(x: torch.Tensor, sampling) -> None:
+    """Virtual samples are [nv, ...] with the per-sample shape of x (same layout)."""
+    if sampling.xv is not None and tuple(sampling.xv.shape[1:]) != tuple(x.shape[1:]):
+        raise TypeError("xv must have the per-sample shape of x")
+
+
 def _vec(t: torch.Tensor, C: int) -> int:
     if t.dtype != torch.float32 or t.numel() != C:
         raise TypeError("per-channel vectors must be float32 of length C")
@@ -282,6 +295,7 @@ def _workspace(x, sampling, workspace):
 # ----------------------------------------------------------------------------- the three calls
 def forward(x, gamma, beta, eps, sampling: Sampling, y=None, mean=None, invstd=None, workspace=None):
     """bns_forward: returns (y, mean, invstd)."""
+    _check_virtual(x, sampling)
     sh, sp = _shape(x), sampling._c()
     C = x.shape[1]
     y = torch.empty_like(x) if y is None else y
@@ -289,7 +303,7 @@ def forward(x, gamma, beta, eps, sampling: Sampling, y=None, mean=None, invstd=N
     invstd = torch.empty(C, dtype=torch.float32, device=x.device) if invstd is None else invstd
     ws, wp, wn = _workspace(x, sampling, workspace)
     st = load().bns_forward(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), ctypes.byref(sp),
-                            _dev(y), _vec(mean, C), _vec(invstd, C), wp, wn, _stream())
+                            _like(y, x, "y"), _vec(mean, C), _vec(invstd, C), wp, wn, _stream())
     _check(st, "bns_forward")
     return y, mean, invstd
 
@@ -302,16 +316,18 @@ def forward_static(x, gamma, beta, eps, sampling: Sampling, y, mean, invstd):
     """bns_forward_static: the forward for callers that may not allocate device memory.  The caller
     passes every tensor, outputs included; the scratch is the array built into the library, shared by
     all calls on the device (so do not overlap two of them).  Returns (y, mean, invstd)."""
+    _check_virtual(x, sampling)
     sh, sp = _shape(x), sampling._c()
     C = x.shape[1]
     st = load().bns_forward_static(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps),
-                                   ctypes.byref(sp), _dev(y), _vec(mean, C), _vec(invstd, C), _stream())
+                                   ctypes.byref(sp), _like(y, x, "y"), _vec(mean, C), _vec(invstd, C), _stream())
     _check(st, "bns_forward_static")
     return y, mean, invstd
 
 
 def backward(x, dy, gamma, mean, invstd, sampling: Sampling, dx=None, dgamma=None, dbeta=None, workspace=None):
     """bns_backward: returns (dx, dgamma, dbeta)."""
+    _check_virtual(x, sampling)
     sh, sp = _shape(x), sampling._c()
     C = x.shape[1]
     if dy.shape != x.shape or dy.dtype != x.dtype:
@@ -321,7 +337,7 @@ def backward(x, dy, gamma, mean, invstd, sampling: Sampling, dx=None, dgamma=Non
     dbeta = torch.empty(C, dtype=torch.float32, device=x.device) if dbeta is None else dbeta
     ws, wp, wn = _workspace(x, sampling, workspace)
     st = load().bns_backward(ctypes.byref(sh), _dev(x), _dev(dy), _vec(gamma, C), _vec(mean, C), _vec(invstd, C),
-                             ctypes.byref(sp), _dev(dx), _vec(dgamma, C), _vec(dbeta, C), wp, wn, _stream())
+                             ctypes.byref(sp), _like(dx, x, "dx"), _vec(dgamma, C), _vec(dbeta, C), wp, wn, _stream())
     _check(st, "bns_backward")
     return dx, dgamma, dbeta
 
@@ -334,7 +350,7 @@ def full_bn(x, gamma, beta, eps, y=None, mean=None, invstd=None, workspace=None)
     mean = torch.empty(C, dtype=torch.float32, device=x.device) if mean is None else mean
     invstd = torch.empty(C, dtype=torch.float32, device=x.device) if invstd is None else invstd
     ws, wp, wn = _workspace(x, Sampling.full(), workspace)
-    st = load().bns_full_bn(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), _dev(y),
+    st = load().bns_full_bn(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), _like(y, x, "y"),
                             _vec(mean, C), _vec(invstd, C), wp, wn, _stream())
     _check(st, "bns_full_bn")
     return y, mean, invstd
@@ -373,7 +389,7 @@ class Prepared:
         self._sh, self._sp = _shape(x), sampling._c()
         self._eps = float(eps)
         self._full = bool(full_bn_entry)
-        self._x, self._dy, self._y, self._dx = _dev(x), _dev(dy), _dev(y), _dev(dx)
+        self._x, self._dy, self._y, self._dx = _dev(x), _dev(dy), _like(y, x, "y"), _like(dx, x, "dx")
         self._gamma, self._beta = _vec(gamma, C), _vec(beta, C)
         self._mean, self._invstd = _vec(mean, C), _vec(invstd, C)
         self._dgamma, self._dbeta = _vec(dgamma, C), _vec(dbeta, C)
@@ -413,6 +429,7 @@ def workspace_bytes_mixed(x, sampling: Sampling) -> int:
 def forward_mixed(x, gamma, beta, eps, mix, sampling: Sampling, workspace=None, y=None, stats=None):
     """bns_forward_mixed: returns (y, mean, invstd, mean_s, mean_v); yv goes to sampling.yv.  `stats` may
     give the four float32[C] output tensors (mean, invstd, mean_s, mean_v)."""
+    _check_virtual(x, sampling)
     sh, sp = _shape(x), sampling._c()
     C = x.shape[1]
     y = torch.empty_like(x) if y is None else y
@@ -421,7 +438,7 @@ def forward_mixed(x, gamma, beta, eps, mix, sampling: Sampling, workspace=None, 
     if workspace is None:
         workspace = torch.empty(workspace_bytes_mixed(x, sampling), dtype=torch.uint8, device=x.device)
     st = load().bns_forward_mixed(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), float(mix),
-                                  ctypes.byref(sp), _dev(y), _vec(mean, C), _vec(invstd, C), _vec(mean_s, C),
+                                  ctypes.byref(sp), _like(y, x, "y"), _vec(mean, C), _vec(invstd, C), _vec(mean_s, C),
                                   _vec(mean_v, C), workspace.data_ptr(), workspace.numel(), _stream())
     _check(st, "bns_forward_mixed")
     return y, mean, invstd, mean_s, mean_v
@@ -430,6 +447,7 @@ def forward_mixed(x, gamma, beta, eps, mix, sampling: Sampling, workspace=None, 
 def backward_mixed(x, dy, gamma, mean, invstd, mean_s, mean_v, mix, sampling: Sampling, workspace=None, dx=None,
                    grads=None):
     """bns_backward_mixed: returns (dx, dgamma, dbeta); dxv goes to sampling.dxv."""
+    _check_virtual(x, sampling)
     sh, sp = _shape(x), sampling._c()
     C = x.shape[1]
     dx = torch.empty_like(x) if dx is None else dx
@@ -438,7 +456,7 @@ def backward_mixed(x, dy, gamma, mean, invstd, mean_s, mean_v, mix, sampling: Sa
     if workspace is None:
         workspace = torch.empty(workspace_bytes_mixed(x, sampling), dtype=torch.uint8, device=x.device)
     st = load().bns_backward_mixed(ctypes.byref(sh), _dev(x), _dev(dy), _vec(gamma, C), _vec(mean, C), _vec(invstd, C),
-                                   _vec(mean_s, C), _vec(mean_v, C), float(mix), ctypes.byref(sp), _dev(dx),
+                                   _vec(mean_s, C), _vec(mean_v, C), float(mix), ctypes.byref(sp), _like(dx, x, "dx"),
                                    _vec(dgamma, C), _vec(dbeta, C), workspace.data_ptr(), workspace.numel(), _stream())
     _check(st, "bns_backward_mixed")
     return dx, dgamma, dbeta
@@ -459,7 +477,7 @@ def inference_forward(x, gamma, beta, eps, mean_ma, var_ma, y=None, workspace=No
     y = torch.empty_like(x) if y is None else y
     ws, wp, wn = _workspace(x, Sampling.full(), workspace)
     st = load().bns_inference_forward(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps),
-                                      _vec(mean_ma, C), _vec(var_ma, C), _dev(y), wp, wn, _stream())
+                                      _vec(mean_ma, C), _vec(var_ma, C), _like(y, x, "y"), wp, wn, _stream())
     _check(st, "bns_inference_forward")
     return y
 
@@ -490,7 +508,7 @@ def sync_normalize(x, gamma, beta, mean, invstd, y=None):
     C = x.shape[1]
     y = torch.empty_like(x) if y is None else y
     _check(load().bns_sync_normalize(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), _vec(mean, C),
-                                     _vec(invstd, C), _dev(y), _stream()), "bns_sync_normalize")
+                                     _vec(invstd, C), _like(y, x, "y"), _stream()), "bns_sync_normalize")
     return y
 
 
@@ -560,6 +578,7 @@ def _shape_nhwc(x: torch.Tensor) -> _Shape:
 def forward_nhwc(x, gamma, beta, eps, sampling: Sampling, workspace=None):
     """bns_forward_nhwc on a dense [N,H,W,C] tensor (virtual tensors in `sampling` are [nv,H,W,C] too);
     returns (y, mean, invstd, workspace) - pass the workspace on to backward_nhwc."""
+    _check_virtual(x, sampling)
     sh, sp = _shape_nhwc(x), sampling._c()
     C = x.shape[3]
     n = load().bns_workspace_bytes_nhwc(ctypes.byref(sh), ctypes.byref(sp))
@@ -578,6 +597,7 @@ def forward_nhwc(x, gamma, beta, eps, sampling: Sampling, workspace=None):
 
 def backward_nhwc(x, dy, gamma, mean, invstd, sampling: Sampling, workspace):
     """bns_backward_nhwc: returns (dx, dgamma, dbeta)."""
+    _check_virtual(x, sampling)
     sh, sp = _shape_nhwc(x), sampling._c()
     C = x.shape[3]
     dx = torch.empty_like(x)
