@@ -111,6 +111,34 @@ struct Vec {
     __device__ __forceinline__ void store(S* p) const { *reinterpret_cast<raw_t*>(p) = raw; }
     __device__ __forceinline__ float get(int j) const { return to_float<T>(reinterpret_cast<const S*>(&raw)[j]); }
     __device__ __forceinline__ void set(int j, float v) { reinterpret_cast<S*>(&raw)[j] = from_float<T>(v); }
+    // whole-vector conversion; the bf16 case works on 32-bit pairs (one shift or mask per element on the
+    // way in, one cvt.rn.bf16x2.f32 per pair on the way out)
+    __device__ __forceinline__ void unpack(float (&f)[V]) const {
+        if constexpr (sizeof(S) == 2 && V >= 2) {
+            const unsigned* w = reinterpret_cast<const unsigned*>(&raw);
+#pragma unroll
+            for (int q = 0; q < V / 2; ++q) {
+                f[2 * q] = __uint_as_float(w[q] << 16);
+                f[2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < V; ++j) f[j] = get(j);
+        }
+    }
+    __device__ __forceinline__ void pack(const float (&f)[V]) {
+        if constexpr (sizeof(S) == 2 && V >= 2) {
+            unsigned* w = reinterpret_cast<unsigned*>(&raw);
+#pragma unroll
+            for (int q = 0; q < V / 2; ++q) {
+                __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * q], f[2 * q + 1]);  // low half = first argument
+                w[q] = *reinterpret_cast<unsigned*>(&h);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < V; ++j) set(j, f[j]);
+        }
+    }
 };
 
 // Channels of the V positions p .. p+V-1 (HW may be smaller than V).
@@ -127,6 +155,19 @@ __device__ __forceinline__ void position_channels(unsigned p, int HW, int (&c)[V
         }
     }
 }
+
+// When a feature map holds at least V positions, the V positions of a thread meet at most two channels:
+// c0 for positions j < jb and c0 + 1 from jb on (jb = V when the thread stays inside one channel).
+struct TwoChannels {
+    int c0, c1, jb;
+    __device__ __forceinline__ TwoChannels(unsigned p, int HW, int V) {
+        c0 = static_cast<int>(p / static_cast<unsigned>(HW));
+        const int r = static_cast<int>(p - static_cast<unsigned>(c0) * static_cast<unsigned>(HW));
+        jb = min(V, HW - r);
+        c1 = jb < V ? c0 + 1 : c0;
+    }
+    __device__ __forceinline__ float pick(int j, float lo, float hi) const { return j < jb ? lo : hi; }
+};
 
 // ------------------------------------------------------------------------------------ moments
 // (count, mean, sum of squared deviations) of a set; merge() is the pairwise update of Chan et al.
@@ -636,7 +677,17 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
     for (int j = 0; j < V; ++j) acc_dy[j] = acc_dyxc[j] = 0.f;
     if (p < P) {
         float a[V], mu[V];
-        {
+        if (HW >= V) {  // at most two channels per thread: two parameter sets, selected per position
+            const TwoChannels ch(p, HW, V);
+            const float mu0 = mean[ch.c0], mu1 = mean[ch.c1];
+            const float a0 = WRITE_DX ? gamma[ch.c0] * invstd[ch.c0] : 0.f;
+            const float a1 = WRITE_DX ? gamma[ch.c1] * invstd[ch.c1] : 0.f;
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                mu[j] = ch.pick(j, mu0, mu1);
+                a[j] = ch.pick(j, a0, a1);
+            }
+        } else {
             int c[V];
             position_channels<V>(p, HW, c);
 #pragma unroll
@@ -660,14 +711,19 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
             }
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
+                float g[V], xv[V];
+                vg[u].unpack(g);
+                vx[u].unpack(xv);
 #pragma unroll
                 for (int j = 0; j < V; ++j) {
-                    float g = vg[u].get(j);
-                    acc_dy[j] += g;
-                    acc_dyxc[j] = fmaf(g, vx[u].get(j) - mu[j], acc_dyxc[j]);
-                    if (WRITE_DX) vg[u].set(j, a[j] * g);
+                    acc_dy[j] += g[j];
+                    acc_dyxc[j] = fmaf(g[j], xv[j] - mu[j], acc_dyxc[j]);
+                    if (WRITE_DX) g[j] *= a[j];
                 }
-                if (WRITE_DX) vg[u].store(op + static_cast<size_t>(row[u]) * P);
+                if (WRITE_DX) {
+                    vg[u].pack(g);
+                    vg[u].store(op + static_cast<size_t>(row[u]) * P);
+                }
             }
         }
         for (; i < order.rows; i += nchunks) {
