@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one col_bwd_reduce_kernel<F32,4,true> launch on the default
 # workload's layer shape (256x64x56x56 fp32), from the ncu capture summarised in
 # profiles/col_bwd_reduce_f32_resnet18_stage1.md; reported only for that workload.
-BWD_REDUCE_DRAM_TRAFFIC_BYTES = 579_660_800   # 411.13 MB read + 168.53 MB written (rest of dx still dirty in L2)
+BWD_REDUCE_DRAM_TRAFFIC_BYTES = 580_750_336   # 411.14 MB read + 169.61 MB written (rest of dx still dirty in L2)
 
 
 # ----------------------------------------------------------------------------- workloads
