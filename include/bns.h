@@ -305,6 +305,24 @@ bns_status bns_debug_selection_mask(const bns_shape* shape, const bns_sampling* 
 #define BNS_FLAG_BAD_OFFSET 1u /* a device-resident patch offset was outside [0,H-ph] x [0,W-pw] */
 bns_status bns_workspace_status(const void* workspace, uint32_t* flags, void* cuda_stream);
 
+/*
+ * The one-launch path.  A layer whose per-channel data (N*H*W elements, twice that in the backward),
+ * split over the up to 8 blocks of a thread-block cluster, fits their shared memory runs its whole
+ * forward, and its whole backward, as one kernel each: the tensor is read from HBM once and written
+ * once, the sampled statistics (Eq. 3) and the sums of Eq. 5 are taken from the on-chip copy and
+ * combined across the cluster in a fixed order.  bns_forward, bns_backward and bns_full_bn choose it
+ * by themselves; results obey the same definition and tolerances as the streaming path.
+ * bns_slab_plan reports the choice for a shape and rule: returns 1 and fills plan[0..5] = channels
+ * per cluster, blocks per cluster, samples per block, shared-memory bytes per block, blocks per
+ * launch, row lanes - or returns 0 when the streaming path is used.  (HOST pointer.)
+ * Those kernels wait for their bulk copies with a bounded number of polls; bns_wait_timeouts
+ * synchronises the stream and returns in *count (HOST) how many such waits have run out on the
+ * current device since the library was loaded.  Anything but 0 means results were computed from
+ * incomplete data.
+ */
+int bns_slab_plan(const bns_shape* shape, const bns_sampling* sampling, int backward, int32_t* plan);
+bns_status bns_wait_timeouts(uint32_t* count, void* cuda_stream);
+
 const char* bns_status_string(bns_status status);
 
 /* ---- measurement hooks (process-wide, not thread-safe; off by default) ---------------------- */
@@ -321,7 +339,9 @@ typedef enum {
     BNS_KERNEL_DIRECT_MOMENTS = 9, /* statistics of a small sampled set, one block per channel    */
     BNS_KERNEL_DIRECT_FIXUP = 10,  /* backward sums combined + statistics terms, small sampled set */
     BNS_KERNEL_VECTOR = 11,        /* C-length kernels: mixing of statistics, moving average          */
-    BNS_KERNEL_KINDS = 12
+    BNS_KERNEL_SLAB_FORWARD = 12,  /* whole forward of a layer whose channel data fits on chip        */
+    BNS_KERNEL_SLAB_BACKWARD = 13, /* whole backward of such a layer                                   */
+    BNS_KERNEL_KINDS = 14
 } bns_kernel_kind;
 
 /* Number of kernels this library has launched in this process since load (or since reset). */
@@ -336,11 +356,14 @@ const char* bns_kernel_name(int kernel_kind);
 
 /* Launch-shape knobs (process-wide; change them only while no call is in flight, and recompute
  * bns_workspace_bytes afterwards).  "target_blocks" / "min_chunk": blocks per launch and least rows
- * per block of the streaming kernels; "stat_target_blocks" / "stat_min_chunk": the same for the
+ * per block of the streaming kernels (0 = a multiple of the SM count); "stat_target_blocks" / "stat_min_chunk": the same for the
  * statistics kernels; "direct_max": sampled elements per channel up to which one block per channel computes the
  * statistics (and, in the backward, combines the sums and applies the statistics terms) without
  * partial sums, 0 = never; "nhwc_blocks": blocks per launch of the channels-last kernels (each block leaves one partial per
- * channel); "pdl": 0/1 programmatic dependent launch; "l2_order": 0/1 visit rows in an
+ * channel); "slab": 0/1 use the one-launch path where it applies, "slab_cta_kb": preferred shared memory per block of
+ * that path in KiB, "slab_min_ctas": grow its clusters while a launch has fewer blocks (0 = two per SM), "slab_max_mb":
+ * tensors above this many MiB keep the streaming path, "slab_cluster_max": largest cluster (1..8);
+ * "pdl": 0/1 programmatic dependent launch; "l2_order": 0/1 visit rows in an
  * order that lets a kernel find in L2 what the previous one read.  Returns BNS_OK,
  * BNS_ERR_RULE for an unknown name or BNS_ERR_SHAPE for a value < 1. */
 int bns_set_tuning(const char* name, int value);

@@ -23,16 +23,16 @@ RULE_FULL, RULE_BATCH, RULE_FEATURE, RULE_VIRTUAL = 0, 1, 2, 3
 OFF_SHARED, OFF_PER_SAMPLE, OFF_PER_MAP = 0, 1, 2
 FLAG_BAD_OFFSET = 1
 
-KERNEL_KINDS = 12
+KERNEL_KINDS = 14
 (KERNEL_COL_MOMENTS, KERNEL_PATCH_MOMENTS, KERNEL_FINALIZE_STATS, KERNEL_NORMALIZE, KERNEL_BWD_REDUCE,
  KERNEL_FINALIZE_BWD, KERNEL_COL_FIXUP, KERNEL_PATCH_FIXUP, KERNEL_MASK, KERNEL_DIRECT_MOMENTS,
- KERNEL_DIRECT_FIXUP, KERNEL_VECTOR) = range(KERNEL_KINDS)
+ KERNEL_DIRECT_FIXUP, KERNEL_VECTOR, KERNEL_SLAB_FORWARD, KERNEL_SLAB_BACKWARD) = range(KERNEL_KINDS)
 
 EXPORTS = [
     "bns_workspace_bytes", "bns_forward", "bns_forward_static", "bns_static_workspace_bytes", "bns_backward", "bns_full_bn", "bns_host_arena_bytes",
     "bns_forward_backward_host", "bns_debug_selection_mask", "bns_workspace_status", "bns_status_string",
     "bns_launch_count", "bns_launch_count_reset", "bns_profile_enable", "bns_profile_read", "bns_kernel_name",
-    "bns_set_tuning",
+    "bns_set_tuning", "bns_slab_plan", "bns_wait_timeouts",
     "bns_workspace_bytes_mixed", "bns_forward_mixed", "bns_backward_mixed", "bns_update_moving_average",
     "bns_inference_forward",
     "bns_sync_local_moments", "bns_sync_merge_moments", "bns_sync_normalize", "bns_sync_backward_sums",
@@ -145,6 +145,10 @@ def load():
     lib.bns_backward_nhwc.argtypes = [shp, vp, vp, vp, vp, vp, smp, vp, vp, vp, vp, sz, vp]
     lib.bns_set_tuning.restype = ctypes.c_int
     lib.bns_set_tuning.argtypes = [ctypes.c_char_p, ctypes.c_int]
+    lib.bns_slab_plan.restype = ctypes.c_int
+    lib.bns_slab_plan.argtypes = [shp, smp, ctypes.c_int, ctypes.POINTER(ctypes.c_int32)]
+    lib.bns_wait_timeouts.restype = ctypes.c_int
+    lib.bns_wait_timeouts.argtypes = [ctypes.POINTER(ctypes.c_uint32), vp]
     _lib = lib
     return lib
 
@@ -194,7 +198,10 @@ class Sampling:
         return Sampling(self.rule, sample_idx=self.sample_idx, ph=self.ph, pw=self.pw, offset_mode=self.offset_mode,
                         offsets=self.offsets, nv=int(xv.shape[0]), xv=xv, yv=yv, dyv=dyv, dxv=dxv)
 
-    def _c(self) -> _Sampling:
+    def _c(self, shape=None) -> _Sampling:
+        """The C struct.  With `shape` (the _Shape of x) the length of device-resident patch offsets is
+        checked against it: the kernels index them by sample (and channel), so a shorter tensor would be
+        read out of bounds."""
         c = _Sampling()
         c.rule = self.rule
         if self.rule == RULE_BATCH:
@@ -208,6 +215,11 @@ class Sampling:
                 off = self.offsets
                 if not (isinstance(off, torch.Tensor) and off.is_cuda and off.dtype == torch.int32 and off.is_contiguous()):
                     raise TypeError("per-sample / per-map offsets must be a contiguous CUDA int32 tensor")
+                if shape is not None:
+                    pairs = shape.N if self.offset_mode == OFF_PER_SAMPLE else shape.N * shape.C
+                    if off.numel() != 2 * pairs:
+                        raise TypeError(f"offsets must hold {pairs} (oh, ow) pairs for this shape and offset mode, "
+                                        f"got {off.numel()} int32 values")
                 c.offsets = off.data_ptr()
         if self.xv is not None:      # the VIRTUAL rule, or a sampling rule combined with virtual samples (Eq. 4)
             c.nv = int(self.xv.shape[0])
@@ -274,7 +286,8 @@ def _check(status: int, what: str):
 
 
 def workspace_bytes(x: torch.Tensor, sampling: Sampling) -> int:
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     n = load().bns_workspace_bytes(ctypes.byref(sh), ctypes.byref(sp))
     if n == 0:
         raise BnsError(-3, "bns_workspace_bytes (invalid shape or sampling rule)")
@@ -296,7 +309,8 @@ def _workspace(x, sampling, workspace):
 def forward(x, gamma, beta, eps, sampling: Sampling, y=None, mean=None, invstd=None, workspace=None):
     """bns_forward: returns (y, mean, invstd)."""
     _check_virtual(x, sampling)
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     C = x.shape[1]
     y = torch.empty_like(x) if y is None else y
     mean = torch.empty(C, dtype=torch.float32, device=x.device) if mean is None else mean
@@ -317,7 +331,8 @@ def forward_static(x, gamma, beta, eps, sampling: Sampling, y, mean, invstd):
     passes every tensor, outputs included; the scratch is the array built into the library, shared by
     all calls on the device (so do not overlap two of them).  Returns (y, mean, invstd)."""
     _check_virtual(x, sampling)
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     C = x.shape[1]
     st = load().bns_forward_static(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps),
                                    ctypes.byref(sp), _like(y, x, "y"), _vec(mean, C), _vec(invstd, C), _stream())
@@ -328,7 +343,8 @@ def forward_static(x, gamma, beta, eps, sampling: Sampling, y, mean, invstd):
 def backward(x, dy, gamma, mean, invstd, sampling: Sampling, dx=None, dgamma=None, dbeta=None, workspace=None):
     """bns_backward: returns (dx, dgamma, dbeta)."""
     _check_virtual(x, sampling)
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     C = x.shape[1]
     if dy.shape != x.shape or dy.dtype != x.dtype:
         raise TypeError("dy must match x")
@@ -358,7 +374,8 @@ def full_bn(x, gamma, beta, eps, y=None, mean=None, invstd=None, workspace=None)
 
 def selection_mask(x, sampling: Sampling, workspace=None):
     """bns_debug_selection_mask: uint8 [N,C,H,W]."""
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     mask = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
     ws, wp, wn = _workspace(x, sampling, workspace)
     _check(load().bns_debug_selection_mask(ctypes.byref(sh), ctypes.byref(sp), mask.data_ptr(), wp, wn, _stream()),
@@ -386,7 +403,8 @@ class Prepared:
             raise TypeError("dy must match x")
         self._keep = (x, dy, gamma, beta, sampling, y, dx, mean, invstd, dgamma, dbeta, workspace)
         self._lib = load()
-        self._sh, self._sp = _shape(x), sampling._c()
+        self._sh = _shape(x)
+        self._sp = sampling._c(self._sh)
         self._eps = float(eps)
         self._full = bool(full_bn_entry)
         self._x, self._dy, self._y, self._dx = _dev(x), _dev(dy), _like(y, x, "y"), _like(dx, x, "dx")
@@ -419,7 +437,8 @@ class Prepared:
 
 # ----------------------------------------------------------------------------- Eq. 4 and Appendix D
 def workspace_bytes_mixed(x, sampling: Sampling) -> int:
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     n = load().bns_workspace_bytes_mixed(ctypes.byref(sh), ctypes.byref(sp))
     if n == 0:
         raise BnsError(-3, "bns_workspace_bytes_mixed (invalid shape or sampling rule)")
@@ -430,7 +449,8 @@ def forward_mixed(x, gamma, beta, eps, mix, sampling: Sampling, workspace=None, 
     """bns_forward_mixed: returns (y, mean, invstd, mean_s, mean_v); yv goes to sampling.yv.  `stats` may
     give the four float32[C] output tensors (mean, invstd, mean_s, mean_v)."""
     _check_virtual(x, sampling)
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     C = x.shape[1]
     y = torch.empty_like(x) if y is None else y
     mean, invstd, mean_s, mean_v = stats if stats is not None else (
@@ -448,7 +468,8 @@ def backward_mixed(x, dy, gamma, mean, invstd, mean_s, mean_v, mix, sampling: Sa
                    grads=None):
     """bns_backward_mixed: returns (dx, dgamma, dbeta); dxv goes to sampling.dxv."""
     _check_virtual(x, sampling)
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     C = x.shape[1]
     dx = torch.empty_like(x) if dx is None else dx
     dgamma, dbeta = grads if grads is not None else (
@@ -485,7 +506,8 @@ def inference_forward(x, gamma, beta, eps, mean_ma, var_ma, y=None, workspace=No
 # ----------------------------------------------------------------------------- statistics shared by several GPUs
 def sync_local_moments(x, sampling: Sampling, eps, workspace=None):
     """bns_sync_local_moments: float32 [3, C] = (count, mean, M2) of this rank's sampled set."""
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     moments = torch.empty(3, x.shape[1], dtype=torch.float32, device=x.device)
     ws, wp, wn = _workspace(x, sampling, workspace)
     _check(load().bns_sync_local_moments(ctypes.byref(sh), _dev(x), ctypes.byref(sp), float(eps), moments.data_ptr(),
@@ -527,7 +549,8 @@ def sync_backward_sums(x, dy, gamma, mean, invstd, dx=None, workspace=None):
 
 def sync_backward_apply(x, dy, gamma, mean, invstd, sampling: Sampling, sums, sampled_total, dx, workspace=None):
     """bns_sync_backward_apply: adds the statistics terms to dx on this rank's sampled elements."""
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     C = x.shape[1]
     ws, wp, wn = _workspace(x, sampling, workspace)
     _check(load().bns_sync_backward_apply(ctypes.byref(sh), _dev(x), _dev(dy), _vec(gamma, C), _vec(mean, C),
@@ -539,7 +562,8 @@ def sync_backward_apply(x, dy, gamma, mean, invstd, sampling: Sampling, sums, sa
 # ----------------------------------------------------------------------------- BN + residual add + ReLU
 def forward_relu(x, residual, gamma, beta, eps, sampling: Sampling, workspace=None):
     """bns_forward_relu: returns (y, mean, invstd) with y = max(0, BN(x) + residual); residual may be None."""
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     C = x.shape[1]
     y = torch.empty_like(x)
     mean, invstd = (torch.empty(C, dtype=torch.float32, device=x.device) for _ in range(2))
@@ -553,7 +577,8 @@ def forward_relu(x, residual, gamma, beta, eps, sampling: Sampling, workspace=No
 
 def backward_relu(x, residual, dy, gamma, beta, mean, invstd, sampling: Sampling, workspace=None):
     """bns_backward_relu: returns (dx, dresidual or None, dgamma, dbeta)."""
-    sh, sp = _shape(x), sampling._c()
+    sh = _shape(x)
+    sp = sampling._c(sh)
     C = x.shape[1]
     dx = torch.empty_like(x)
     dres = None if residual is None else torch.empty_like(x)
@@ -579,7 +604,8 @@ def forward_nhwc(x, gamma, beta, eps, sampling: Sampling, workspace=None):
     """bns_forward_nhwc on a dense [N,H,W,C] tensor (virtual tensors in `sampling` are [nv,H,W,C] too);
     returns (y, mean, invstd, workspace) - pass the workspace on to backward_nhwc."""
     _check_virtual(x, sampling)
-    sh, sp = _shape_nhwc(x), sampling._c()
+    sh = _shape_nhwc(x)
+    sp = sampling._c(sh)
     C = x.shape[3]
     n = load().bns_workspace_bytes_nhwc(ctypes.byref(sh), ctypes.byref(sp))
     if n == 0:
@@ -598,7 +624,8 @@ def forward_nhwc(x, gamma, beta, eps, sampling: Sampling, workspace=None):
 def backward_nhwc(x, dy, gamma, mean, invstd, sampling: Sampling, workspace):
     """bns_backward_nhwc: returns (dx, dgamma, dbeta)."""
     _check_virtual(x, sampling)
-    sh, sp = _shape_nhwc(x), sampling._c()
+    sh = _shape_nhwc(x)
+    sp = sampling._c(sh)
     C = x.shape[3]
     dx = torch.empty_like(x)
     dgamma, dbeta = (torch.empty(C, dtype=torch.float32, device=x.device) for _ in range(2))
@@ -613,7 +640,7 @@ def backward_nhwc(x, dy, gamma, mean, invstd, sampling: Sampling, workspace):
 def host_arena_bytes(shape, dtype, sampling: Sampling) -> int:
     N, C, H, W = shape
     sh = _Shape(N, C, H, W, F32 if dtype == torch.float32 else BF16)
-    sp = sampling._c()
+    sp = sampling._c(sh)
     return int(load().bns_host_arena_bytes(ctypes.byref(sh), ctypes.byref(sp)))
 
 
@@ -657,6 +684,24 @@ def profile_read(kind: int):
 def set_tuning(name: str, value: int) -> None:
     """bns_set_tuning: launch-shape knobs (see include/bns.h)."""
     _check(load().bns_set_tuning(name.encode(), int(value)), f"bns_set_tuning({name})")
+
+
+def slab_plan(x: torch.Tensor, sampling: Sampling, backward: bool = False):
+    """bns_slab_plan: None when the streaming path serves this shape and rule, else a dict describing the
+    one-launch path (channels and blocks per cluster, samples and shared-memory bytes per block, grid)."""
+    sh = _shape(x)
+    sp = sampling._c(sh)
+    out = (ctypes.c_int32 * 6)()
+    if not load().bns_slab_plan(ctypes.byref(sh), ctypes.byref(sp), 1 if backward else 0, out):
+        return None
+    return dict(zip(("channels", "cluster", "rows", "smem_bytes", "grid", "row_lanes"), (int(v) for v in out)))
+
+
+def wait_timeouts() -> int:
+    """bns_wait_timeouts: bounded waits that ran out on this device since the library was loaded."""
+    n = ctypes.c_uint32(0)
+    _check(load().bns_wait_timeouts(ctypes.byref(n), _stream()), "bns_wait_timeouts")
+    return int(n.value)
 
 
 def kernel_name(kind: int) -> str:

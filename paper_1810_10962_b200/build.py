@@ -9,7 +9,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIBRARY = os.path.join(HERE, "libbns.so")
 SOURCES = [os.path.join(CSRC, "bns_api.cu")]
-HEADERS = [os.path.join(CSRC, "bns_kernels.cuh"), os.path.join(CSRC, "bns_nhwc_kernels.cuh"), os.path.join(ROOT, "include", "bns.h")]
+HEADERS = [os.path.join(CSRC, "bns_kernels.cuh"), os.path.join(CSRC, "bns_nhwc_kernels.cuh"), os.path.join(CSRC, "bns_slab_kernels.cuh"), os.path.join(ROOT, "include", "bns.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

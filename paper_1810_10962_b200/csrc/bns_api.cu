@@ -11,6 +11,7 @@
 
 #include "bns_kernels.cuh"
 #include "bns_nhwc_kernels.cuh"
+#include "bns_slab_kernels.cuh"
 
 namespace {
 
@@ -18,7 +19,23 @@ using namespace bns;
 
 constexpr size_t kAlign = 256;
 constexpr size_t kHeaderBytes = 256;  // status word lives at the start of the workspace
-constexpr int kSmCount = 148;
+constexpr int kMaxDevices = 64;
+constexpr int kSmCountFallback = 148;     // B200; used only if the device cannot be queried
+
+// Streaming multiprocessors of the current device (queried once per device).
+int sm_count() {
+    static std::atomic<int> cached[kMaxDevices];
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return kSmCountFallback;
+    int n = cached[device].load(std::memory_order_relaxed);
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        return kSmCountFallback;
+    }
+    cached[device].store(n, std::memory_order_relaxed);
+    return n;
+}
 
 size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 int elem_bytes(int dtype) { return dtype == BNS_F32 ? 4 : 2; }
@@ -81,13 +98,18 @@ struct ColPlan {
     size_t partial_count() const { return static_cast<size_t>(nchunks) * tiles * max_slots; }
 };
 
-int g_target_blocks = kSmCount * 32;      // streaming kernels: blocks per launch aimed at when splitting the rows
+// Blocks per launch aimed at when splitting the rows; 0 = a multiple of the SM count (32 per SM for the
+// streaming kernels, 8 per SM - one wave, all loads in flight - for the short statistics kernels).
+int g_target_blocks = 0;
 int g_min_chunk = 8;                      // ... but at least this many rows per block
-int g_stat_target_blocks = kSmCount * 8;  // short statistics kernels: one wave of blocks, all loads in flight
+int g_stat_target_blocks = 0;
 int g_stat_min_chunk = 1;
 
+int target_blocks_streaming() { return g_target_blocks > 0 ? g_target_blocks : sm_count() * 32; }
+int target_blocks_statistics() { return g_stat_target_blocks > 0 ? g_stat_target_blocks : sm_count() * 8; }
+
 ColPlan plan_col(unsigned P, int HW, int C, int rows, int ebytes, bool statistics = false) {
-    const int target_blocks = statistics ? g_stat_target_blocks : g_target_blocks;
+    const int target_blocks = statistics ? target_blocks_statistics() : target_blocks_streaming();
     const int min_chunk = statistics ? g_stat_min_chunk : g_min_chunk;
     ColPlan pl;
     int V = 16 / ebytes;
@@ -120,12 +142,105 @@ PatchPlan plan_patch(int N, int C, int ph, int pw) {
     const long PP = static_cast<long>(ph) * pw;
     const long Pc = static_cast<long>(C) * PP;
     pl.tiles = static_cast<unsigned>((Pc + kThreads - 1) / kThreads);
-    long want = g_stat_target_blocks / static_cast<long>(pl.tiles);
+    long want = target_blocks_statistics() / static_cast<long>(pl.tiles);
     long nchunks = std::max(1L, std::min<long>(want, std::max(1, N / 4)));
     pl.chunk = static_cast<int>((N + nchunks - 1) / nchunks);
     pl.nchunks = (N + pl.chunk - 1) / pl.chunk;
     pl.max_slots = static_cast<int>(std::min<long>((kThreads + PP - 2) / PP + 1, C));
     return pl;
+}
+
+// ------------------------------------------------------------------------------------ slab (on-chip) path
+// A layer takes the one-launch path when the data of a channel group, split over the blocks of a
+// cluster, fits their shared memory (see bns_slab_kernels.cuh).
+struct SlabPlan {
+    bool ok = false;
+    SlabGeom geo{};
+    unsigned grid = 0;
+};
+
+bool g_slab = true;            // use the one-launch path where it applies
+int g_slab_cta_kb = 112;       // preferred shared memory per block: two blocks per SM stay resident
+int g_slab_min_ctas = 0;       // grow the cluster while the launch has fewer blocks than this; 0 = 2 per SM
+int g_slab_max_mb = 1 << 20;   // tensors larger than this many MiB keep the streaming path
+int g_slab_cluster_max = 8;    // largest cluster (8 is the portable limit)
+constexpr size_t kSlabSmemLimit = 227 * 1024;  // most dynamic shared memory a block may ask for
+
+size_t gcd_size(size_t a, size_t b) { return b ? gcd_size(b, a % b) : a; }
+
+// Shared memory layout of one block for cluster size R; returns the total bytes.
+size_t slab_layout(SlabGeom& g, int R, int tensors, int origin_stride) {
+    auto up = [](size_t v, size_t a) { return (v + a - 1) / a * a; };
+    g.R = R;
+    g.rows_max = (g.N + R - 1) / R;
+    const int K = tensors;  // accumulators per position: 1 forward (one sum at a time), 2 backward
+    size_t off = 128;       // the copy barrier lives at offset 0
+    g.off_x = static_cast<unsigned>(off);
+    off = up(off + static_cast<size_t>(g.rows_max) * g.row_bytes, 128);
+    g.off_g = static_cast<unsigned>(off);
+    if (tensors == 2) off = up(off + static_cast<size_t>(g.rows_max) * g.row_bytes, 128);
+    g.off_fold = static_cast<unsigned>(off);
+    off = up(off + static_cast<size_t>(K) * g.RL * g.Wd * sizeof(float), 16);
+    g.off_slices = static_cast<unsigned>(off);
+    off = up(off + static_cast<size_t>(std::max(g.G, kWarps)) * K * sizeof(float), 16);
+    g.off_part = static_cast<unsigned>(off);
+    off = up(off + static_cast<size_t>(g.G) * 16, 16);
+    g.off_coef = static_cast<unsigned>(off);
+    off = up(off + static_cast<size_t>(g.G) * 16, 16);
+    g.off_flag = static_cast<unsigned>(off);
+    off = up(off + static_cast<size_t>(g.rows_max), 16);
+    g.off_origin = static_cast<unsigned>(off);
+    off = up(off + static_cast<size_t>(g.rows_max) * origin_stride * sizeof(int2), 16);
+    g.total_bytes = static_cast<unsigned>(off);
+    return off;
+}
+
+// origin_stride: 0 = no device-resident patch offsets, 1 = one pair per sample, 2 = one pair per map
+SlabPlan plan_slab(int N, int C, int H, int W, int ebytes, bool backward, int offsets_kind) {
+    SlabPlan sp;
+    if (!g_slab) return sp;
+    const size_t HW = static_cast<size_t>(H) * W;
+    if (H >= 32768 || W >= 65536) return sp;
+    if (static_cast<double>(N) * C * HW * ebytes > static_cast<double>(g_slab_max_mb) * 1048576.0) return sp;
+    const int V = 16 / ebytes;
+    int G = static_cast<int>(16 / gcd_size(HW * ebytes, 16));  // fewest channels whose row segment is a multiple of 16 bytes
+    if (C % G != 0) return sp;
+    while (static_cast<size_t>(G) * HW * ebytes < 512 && C % (2 * G) == 0 && 2 * G * HW / V <= static_cast<size_t>(kThreads) &&
+           2 * G <= 64)
+        G *= 2;
+    if (G * HW / V > static_cast<size_t>(kThreads) || G > kThreads) return sp;
+    SlabGeom& g = sp.geo;
+    g.N = N;
+    g.C = C;
+    g.H = H;
+    g.W = W;
+    g.HW = static_cast<int>(HW);
+    g.G = G;
+    g.Wd = static_cast<int>(G * HW);
+    g.NV = g.Wd / V;
+    g.RL = kThreads / g.NV;
+    g.P = static_cast<unsigned>(C * HW);
+    g.row_bytes = static_cast<unsigned>(g.Wd * ebytes);
+    const int tensors = backward ? 2 : 1;
+    const int stride = offsets_kind == 2 ? G : offsets_kind == 1 ? 1 : 0;
+    const int groups = C / G;
+    const int r_max = std::min(g_slab_cluster_max, N);
+    int R = 0;
+    for (int limit_pass = 0; limit_pass < 2 && !R; ++limit_pass) {
+        const size_t limit = limit_pass == 0 ? std::min(static_cast<size_t>(g_slab_cta_kb) * 1024, kSlabSmemLimit) : kSlabSmemLimit;
+        for (int r = 1; r <= r_max; r *= 2)
+            if (slab_layout(g, r, tensors, stride) <= limit) {
+                R = r;
+                break;
+            }
+    }
+    if (!R) return sp;
+    const int want = g_slab_min_ctas > 0 ? g_slab_min_ctas : 2 * sm_count();
+    while (2 * R <= r_max && groups * R < want && N / (2 * R) >= 4) R *= 2;
+    slab_layout(g, R, tensors, stride);
+    sp.grid = static_cast<unsigned>(groups) * R;
+    sp.ok = true;
+    return sp;
 }
 
 struct Problem {
@@ -143,6 +258,7 @@ struct Problem {
     ColPlan main_plan;             // all N rows of x (normalise, backward pass 1, full statistics, full backward)
     ColPlan stat_plan;             // BATCH: the k sampled rows;  VIRTUAL: the nv rows of xv
     PatchPlan patch_plan;
+    SlabPlan slab_fwd, slab_bwd;   // the one-launch path, when the layer qualifies
     // workspace layout
     size_t off_list, off_stats, off_bwd, off_bwd_v, total;
 };
@@ -244,6 +360,9 @@ bns_status make_problem(const bns_shape* sh, const bns_sampling* sp, Problem& pb
     pb.off_bwd_v = off;
     if (sp->rule == BNS_RULE_VIRTUAL) off += align_up(pb.stat_plan.partial_count() * sizeof(float2));
     pb.total = off;
+    const int offsets_kind = (sp->rule == BNS_RULE_FEATURE && pb.patch.offsets) ? (pb.patch.stride_c ? 2 : 1) : 0;
+    pb.slab_fwd = plan_slab(pb.N, pb.C, pb.H, pb.W, eb, false, offsets_kind);
+    pb.slab_bwd = plan_slab(pb.N, pb.C, pb.H, pb.W, eb, true, offsets_kind);
     return BNS_OK;
 }
 
@@ -257,7 +376,23 @@ T* ws_at(void* ws, size_t off) {
     return reinterpret_cast<T*>(static_cast<char*>(ws) + off);
 }
 
-bns_status last_error() { return cudaGetLastError() == cudaSuccess ? BNS_OK : BNS_ERR_CUDA; }
+// Launch failures of the current call, on this host thread: every launch helper records the return code
+// of its own cudaLaunchKernelEx, so an error that some other code left in the runtime is neither
+// reported as ours nor cleared.
+thread_local bool t_launch_failed = false;
+
+void note_launch(cudaError_t err) {
+    if (err != cudaSuccess) {
+        t_launch_failed = true;
+        cudaGetLastError();  // a failed launch leaves its error behind: take it back out
+    }
+}
+
+bns_status last_error() {
+    const bool failed = t_launch_failed;
+    t_launch_failed = false;
+    return failed ? BNS_ERR_CUDA : BNS_OK;
+}
 
 // Copies a non-contiguous sample list into the workspace; returns the device list or NULL.
 bns_status stage_list(const Problem& pb, const bns_sampling* sp, void* ws, cudaStream_t stream, const int** list) {
@@ -298,7 +433,7 @@ void launch_with(bool early_scheduling, int kind, void (*kernel)(KArgs...), unsi
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = (g_pdl && early_scheduling) ? 1 : 0;
-    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    note_launch(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
 }
 
 // Normal launch of this library: the kernel may be scheduled while its predecessor drains.
@@ -374,6 +509,100 @@ SampleSet sample_set(const Problem& pb, const int* list) {
     return set;
 }
 
+// Launch of a slab kernel: a cluster of `cluster` blocks per channel group and `smem` bytes of dynamic
+// shared memory per block.  The first launch of each kernel on a device raises its shared-memory limit.
+std::mutex g_slab_attr_mutex;
+
+template <typename... KArgs, typename... Args>
+void launch_cluster(int kind, void (*kernel)(KArgs...), unsigned grid, unsigned cluster, size_t smem, cudaStream_t s,
+                    Args&&... args) {
+    {
+        static bool raised[kMaxDevices] = {};  // one array per kernel instantiation
+        int device = -1;
+        if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) {
+            note_launch(cudaErrorInvalidDevice);
+            return;
+        }
+        std::lock_guard<std::mutex> guard(g_slab_attr_mutex);
+        if (!raised[device]) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSlabSmemLimit)) !=
+                cudaSuccess) {
+                note_launch(cudaErrorInvalidValue);
+                return;
+            }
+            raised[device] = true;
+        }
+    }
+    LaunchScope scope(kind, s);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_pdl ? 2 : 1;
+    note_launch(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+}
+
+SlabSel slab_selection(const Problem& pb, const bns_sampling* sp, const int* list) {
+    SlabSel sel{};
+    sel.rule = pb.rule;
+    sel.list = list;
+    sel.begin = pb.rule == BNS_RULE_BATCH ? pb.begin : 0;
+    sel.count = pb.count;
+    sel.patch = pb.patch;
+    sel.inv_s = static_cast<float>(1.0 / pb.s);
+    if (pb.rule == BNS_RULE_VIRTUAL) {
+        sel.nv = sp->nv;
+        sel.xv_is_bf16 = sp->xv_dtype == BNS_BF16;
+        sel.xv = sp->xv;
+        sel.yv = sp->yv;
+        sel.dyv = sp->dyv;
+        sel.dxv = sp->dxv;
+    }
+    return sel;
+}
+
+bns_status slab_forward(const Problem& pb, const bns_sampling* sp, const void* x, const float* gamma, const float* beta,
+                        float eps, void* y, float* mean, float* invstd, void* ws, cudaStream_t stream) {
+    unsigned* status;
+    bns_status st = clear_status(pb, ws, stream, &status);
+    if (st != BNS_OK) return st;
+    const int* list = nullptr;
+    st = stage_list(pb, sp, ws, stream, &list);
+    if (st != BNS_OK) return st;
+    const SlabPlan& pl = pb.slab_fwd;
+    const SlabSel sel = slab_selection(pb, sp, list);
+    BNS_BY_TYPE(pb.dtype, (launch_cluster(BNS_KERNEL_SLAB_FORWARD, slab_forward_kernel<T>, pl.grid, pl.geo.R,
+                                          pl.geo.total_bytes, stream, in<T>(x), out<T>(y), gamma, beta, eps, pl.geo, sel, mean,
+                                          invstd, status)));
+    return last_error();
+}
+
+bns_status slab_backward(const Problem& pb, const bns_sampling* sp, const void* x, const void* dy, const float* gamma,
+                         const float* mean, const float* invstd, void* dx, float* dgamma, float* dbeta, void* ws,
+                         cudaStream_t stream) {
+    unsigned* status;
+    bns_status st = clear_status(pb, ws, stream, &status);
+    if (st != BNS_OK) return st;
+    const int* list = nullptr;
+    st = stage_list(pb, sp, ws, stream, &list);
+    if (st != BNS_OK) return st;
+    const SlabPlan& pl = pb.slab_bwd;
+    const SlabSel sel = slab_selection(pb, sp, list);
+    BNS_BY_TYPE(pb.dtype, (launch_cluster(BNS_KERNEL_SLAB_BACKWARD, slab_backward_kernel<T>, pl.grid, pl.geo.R,
+                                          pl.geo.total_bytes, stream, in<T>(x), in<T>(dy), out<T>(dx), gamma, mean, invstd,
+                                          pl.geo, sel, dgamma, dbeta, status)));
+    return last_error();
+}
+
 // Statistics of the rule's sampled set into mean / invstd: partial moments, then one warp per channel.
 bns_status run_statistics(const Problem& pb, const bns_sampling* sp, const void* x, float eps, float* mean,
                           float* invstd, void* ws, cudaStream_t stream) {
@@ -421,6 +650,7 @@ bns_status run_statistics(const Problem& pb, const bns_sampling* sp, const void*
 
 bns_status forward_impl(const Problem& pb, const bns_sampling* sp, const void* x, const float* gamma, const float* beta,
                         float eps, void* y, float* mean, float* invstd, void* ws, cudaStream_t stream) {
+    if (pb.slab_fwd.ok) return slab_forward(pb, sp, x, gamma, beta, eps, y, mean, invstd, ws, stream);
     bns_status st = run_statistics(pb, sp, x, eps, mean, invstd, ws, stream);
     if (st != BNS_OK) return st;
     const ColPlan& pl = pb.main_plan;
@@ -445,6 +675,7 @@ bns_status forward_impl(const Problem& pb, const bns_sampling* sp, const void* x
 bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* x, const void* dy, const float* gamma,
                          const float* mean, const float* invstd, void* dx, float* dgamma, float* dbeta, void* ws,
                          cudaStream_t stream) {
+    if (pb.slab_bwd.ok) return slab_backward(pb, sp, x, dy, gamma, mean, invstd, dx, dgamma, dbeta, ws, stream);
     const ColPlan& pl = pb.main_plan;
     const ColPlan& pv = pb.stat_plan;
     const bool full = pb.rule == BNS_RULE_FULL;
@@ -649,7 +880,7 @@ bns_status backward_mixed_impl(const MixedProblem& mp, const bns_sampling* sp, c
 }
 
 // ------------------------------------------------------------------------------------ channels-last (NHWC)
-int g_nhwc_blocks = kSmCount * 8;  // blocks per channels-last launch
+int g_nhwc_blocks = 0;  // blocks per channels-last launch; 0 = 8 per SM
 
 struct NhwcLaunch {
     NhwcShape shape;
@@ -672,7 +903,7 @@ NhwcLaunch plan_nhwc(int C, int ebytes, long total, bool statistics) {
     // few, long-lived blocks: every block leaves one partial per channel, so the block count is also the
     // number of partials the finalize kernels have to read per channel
     (void)statistics;
-    const long target = std::max(1L, static_cast<long>(g_nhwc_blocks) / gy);
+    const long target = std::max(1L, static_cast<long>(g_nhwc_blocks > 0 ? g_nhwc_blocks : sm_count() * 8) / gy);
     long rpb = std::max<long>(static_cast<long>(s.RL) * kUnroll * 2, (total + target - 1) / target);
     rpb = (rpb + s.RL - 1) / s.RL * s.RL;
     s.rows_per_block = static_cast<int>(rpb);
@@ -771,7 +1002,7 @@ void launch_grid_block(int kind, void (*kernel)(KArgs...), dim3 grid, int thread
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g_pdl ? 1 : 0;
-    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    note_launch(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
 }
 
 template <typename... KArgs, typename... Args>
@@ -1022,10 +1253,9 @@ bns_status bns_debug_selection_mask(const bns_shape* shape, const bns_sampling* 
     unsigned* status;
     st = clear_status(pb, workspace, stream, &status);
     if (st != BNS_OK) return st;
-    const size_t blocks = std::min<size_t>((pb.elems + kThreads - 1) / kThreads, static_cast<size_t>(kSmCount) * 32);
-    LaunchScope scope(BNS_KERNEL_MASK, stream);
-    selection_mask_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
-        mask, pb.rule, list, pb.begin, pb.count, pb.patch, pb.N, pb.C, pb.H, pb.W, status);
+    const size_t blocks = std::min<size_t>((pb.elems + kThreads - 1) / kThreads, static_cast<size_t>(sm_count()) * 32);
+    launch_after_predecessor(BNS_KERNEL_MASK, selection_mask_kernel, static_cast<unsigned>(blocks), stream, mask, pb.rule,
+                             list, pb.begin, pb.count, pb.patch, pb.N, pb.C, pb.H, pb.W, status);
     return last_error();
 }
 
@@ -1085,17 +1315,25 @@ int bns_set_tuning(const char* name, int value) {
         const char* name;
         int* ivalue;
         bool* bvalue;
-    } knobs[] = {{"target_blocks", &g_target_blocks, nullptr},   {"min_chunk", &g_min_chunk, nullptr},
-                 {"stat_target_blocks", &g_stat_target_blocks, nullptr}, {"stat_min_chunk", &g_stat_min_chunk, nullptr},
-                 {"direct_max", &g_direct_max, nullptr},         {"nhwc_blocks", &g_nhwc_blocks, nullptr},         {"pdl", nullptr, &g_pdl},                       {"l2_order", nullptr, &g_l2_order}};
+        bool zero_allowed;  // 0 has a meaning of its own for this knob (automatic, or never)
+    } knobs[] = {{"target_blocks", &g_target_blocks, nullptr, true},
+                 {"min_chunk", &g_min_chunk, nullptr, false},
+                 {"stat_target_blocks", &g_stat_target_blocks, nullptr, true},
+                 {"stat_min_chunk", &g_stat_min_chunk, nullptr, false},
+                 {"direct_max", &g_direct_max, nullptr, true},
+                 {"nhwc_blocks", &g_nhwc_blocks, nullptr, true},
+                 {"slab", nullptr, &g_slab, false},
+                 {"slab_cta_kb", &g_slab_cta_kb, nullptr, false},
+                 {"slab_min_ctas", &g_slab_min_ctas, nullptr, true},
+                 {"slab_max_mb", &g_slab_max_mb, nullptr, false},
+                 {"slab_cluster_max", &g_slab_cluster_max, nullptr, false},
+                 {"pdl", nullptr, &g_pdl, false},
+                 {"l2_order", nullptr, &g_l2_order, false}};
     for (const Knob& k : knobs) {
         if (std::strcmp(name, k.name) != 0) continue;
         if (k.ivalue) {
-            if (k.ivalue == &g_direct_max && value == 0) {
-                g_direct_max = 0;
-                return BNS_OK;
-            }
-            if (value < 1) return BNS_ERR_SHAPE;
+            if (value < (k.zero_allowed ? 0 : 1)) return BNS_ERR_SHAPE;
+            if (k.ivalue == &g_slab_cluster_max && value > 8) return BNS_ERR_SHAPE;  // 8 is the portable cluster limit
             *k.ivalue = value;
         } else {
             *k.bvalue = value != 0;
@@ -1103,6 +1341,29 @@ int bns_set_tuning(const char* name, int value) {
         return BNS_OK;
     }
     return BNS_ERR_RULE;
+}
+
+int bns_slab_plan(const bns_shape* shape, const bns_sampling* sampling, int backward, int32_t* plan) {
+    Problem pb;
+    if (!plan) return 0;
+    if (make_problem(shape, sampling, pb) != BNS_OK) return 0;
+    const SlabPlan& pl = backward ? pb.slab_bwd : pb.slab_fwd;
+    if (!pl.ok) return 0;
+    plan[0] = pl.geo.G;
+    plan[1] = pl.geo.R;
+    plan[2] = pl.geo.rows_max;
+    plan[3] = static_cast<int32_t>(pl.geo.total_bytes);
+    plan[4] = static_cast<int32_t>(pl.grid);
+    plan[5] = pl.geo.RL;
+    return 1;
+}
+
+bns_status bns_wait_timeouts(uint32_t* count, void* cuda_stream) {
+    if (!count) return BNS_ERR_NULL;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyFromSymbolAsync(count, g_wait_timeouts, sizeof(uint32_t), 0, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return BNS_ERR_CUDA;
+    return cudaStreamSynchronize(stream) == cudaSuccess ? BNS_OK : BNS_ERR_CUDA;
 }
 
 const char* bns_kernel_name(int kernel_kind) {
@@ -1119,6 +1380,8 @@ const char* bns_kernel_name(int kernel_kind) {
     case BNS_KERNEL_DIRECT_MOMENTS: return "direct_moments_kernel";
     case BNS_KERNEL_DIRECT_FIXUP: return "direct_finalize_fixup_kernel";
     case BNS_KERNEL_VECTOR: return "per-channel vector kernels";
+    case BNS_KERNEL_SLAB_FORWARD: return "slab_forward_kernel";
+    case BNS_KERNEL_SLAB_BACKWARD: return "slab_backward_kernel";
     }
     return "unknown";
 }
@@ -1419,7 +1682,6 @@ bns_status bns_backward_nhwc(const bns_shape* shape, const void* x, const void* 
 static __device__ __align__(256) unsigned char g_static_workspace[BNS_STATIC_WORKSPACE_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 void* g_static_workspace_address[kMaxDevices] = {};  // resolved by the first call made on each device
 
 // Device address of the static scratch on the device that is current now.

@@ -127,6 +127,7 @@ def run_gpu(case: Case, use_full_bn_entry=False) -> GpuResult:
         y, mean, invstd = bns.forward(x, gamma, beta, case.eps, sp, workspace=ws)
     dx, dgamma, dbeta = bns.backward(x, dy, gamma, mean, invstd, sp, workspace=ws)
     torch.cuda.synchronize()
+    assert bns.wait_timeouts() == 0, "a bounded wait of a kernel ran out"
     res = GpuResult(_to_host(y), mean.cpu().numpy(), invstd.cpu().numpy(), _to_host(dx), dgamma.cpu().numpy(),
                     dbeta.cpu().numpy(), raw=dict(y=y, mean=mean, invstd=invstd, dx=dx, dgamma=dgamma, dbeta=dbeta))
     if case.rule == "virtual":

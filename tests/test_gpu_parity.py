@@ -10,6 +10,16 @@ from helpers import Case, compare, gpu_sampling, make_case, run_gpu, _to_device
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(autouse=True, params=["onchip", "streaming"])
+def execution_path(request):
+    """Every case runs twice: with the one-launch on-chip path allowed (layers that qualify take it,
+    the others stream anyway) and with it switched off (everything streams)."""
+    from paper_1810_10962_b200 import bns
+    bns.set_tuning("slab", 1 if request.param == "onchip" else 0)
+    yield request.param
+    bns.set_tuning("slab", 1)
+
+
 # ----------------------------------------------------------------------------- config 1: tiny
 @pytest.mark.parametrize("rule,kw", [
     ("batch", dict(k=2, contiguous=False)),
@@ -214,8 +224,8 @@ def test_other_grid_shapes_still_match_the_oracle(target):
             case = make_case(70, 12, 33, 31, rule, seed=86, **kw)
             compare(case, run_gpu(case))
     finally:
-        bns.set_tuning("target_blocks", 148 * 32)
-        bns.set_tuning("stat_target_blocks", 148 * 8)
+        bns.set_tuning("target_blocks", 0)
+        bns.set_tuning("stat_target_blocks", 0)
 
 
 @pytest.mark.parametrize("rule,kw", [
@@ -312,3 +322,63 @@ def test_host_buffer_entry_point(rule, kw, dtype):
     tensor_close(_to_host(dx), b.dx, "dx")
     close_f32(dgamma.numpy(), b.dgamma, "dgamma")
     close_f32(dbeta.numpy(), b.dbeta, "dbeta")
+
+
+# ----------------------------------------------------------------------------- the one-launch on-chip path
+def _device_case(case):
+    import torch
+    x, dy = _to_device(case.x, case.dtype), _to_device(case.dy, case.dtype)
+    gamma, beta = torch.from_numpy(case.gamma).cuda(), torch.from_numpy(case.beta).cuda()
+    return x, dy, gamma, beta
+
+
+@pytest.mark.parametrize("dims,dtype,rule,kw", [
+    ((8, 16, 8, 8), "f32", "batch", dict(k=2)),
+    ((128, 16, 32, 32), "f32", "feature", dict(ph=4, pw=4)),
+    ((128, 32, 16, 16), "f32", "feature", dict(ph=4, pw=4, offset_mode=2)),
+    ((128, 64, 8, 8), "f32", "full", dict()),
+    ((256, 128, 28, 28), "bf16", "virtual", dict(nv=2, with_dyv=False)),
+    ((256, 256, 14, 14), "bf16", "feature", dict(ph=1, pw=1)),
+    ((256, 512, 7, 7), "bf16", "full", dict()),
+])
+def test_qualifying_layers_take_one_launch_per_direction(dims, dtype, rule, kw, execution_path):
+    """Layers whose channel data fits the shared memory of a cluster run forward and backward as one
+    kernel each; with the path switched off the same call takes the streaming kernels."""
+    from paper_1810_10962_b200 import bns
+    case = make_case(*dims, rule, seed=90, dtype=dtype, **kw)
+    x, dy, gamma, beta = _device_case(case)
+    sp = gpu_sampling(case)
+    plans = bns.slab_plan(x, sp, backward=False), bns.slab_plan(x, sp, backward=True)
+    ws = bns.new_workspace(x, sp)
+    before = bns.launch_count()
+    y, mean, invstd = bns.forward(x, gamma, beta, case.eps, sp, workspace=ws)
+    bns.backward(x, dy, gamma, mean, invstd, sp, workspace=ws)
+    launched = bns.launch_count() - before
+    if execution_path == "onchip":
+        assert plans[0] is not None and plans[1] is not None
+        assert plans[0]["cluster"] <= 8 and plans[1]["smem_bytes"] <= 227 * 1024
+        assert launched == 2
+    else:
+        assert plans == (None, None)
+        assert launched >= 4
+    assert bns.wait_timeouts() == 0
+
+
+@pytest.mark.parametrize("cluster_max", [1, 2, 4, 8])
+@pytest.mark.parametrize("rule,kw", [
+    ("batch", dict(k=5, contiguous=False)), ("feature", dict(ph=3, pw=2, offset_mode=1)), ("virtual", dict(nv=2)),
+    ("full", dict()),
+])
+def test_every_cluster_size_matches_the_oracle(cluster_max, rule, kw, execution_path):
+    """The combine across the blocks of a cluster, for 1 to 8 blocks; 37 samples split unevenly."""
+    from paper_1810_10962_b200 import bns
+    if execution_path != "onchip":
+        pytest.skip("cluster sizes only exist on the on-chip path")
+    case = make_case(37, 24, 10, 10, rule, seed=91, **kw)
+    try:
+        bns.set_tuning("slab_cluster_max", cluster_max)
+        bns.set_tuning("slab_min_ctas", 1 << 20)        # always grow the cluster to the limit
+        compare(case, run_gpu(case))
+    finally:
+        bns.set_tuning("slab_cluster_max", 8)
+        bns.set_tuning("slab_min_ctas", 0)
