@@ -173,7 +173,7 @@ size_t slab_layout(SlabGeom& g, int R, int tensors, int origin_stride) {
     auto up = [](size_t v, size_t a) { return (v + a - 1) / a * a; };
     g.R = R;
     g.rows_max = (g.N + R - 1) / R;
-    const int K = tensors;  // accumulators per position: 1 forward (one sum at a time), 2 backward
+    const int K = 2;        // sums kept per position
     size_t off = 128;       // the copy barrier lives at offset 0
     g.off_x = static_cast<unsigned>(off);
     off = up(off + static_cast<size_t>(g.rows_max) * g.row_bytes, 128);
@@ -185,12 +185,14 @@ size_t slab_layout(SlabGeom& g, int R, int tensors, int origin_stride) {
     off = up(off + static_cast<size_t>(std::max(g.G, kWarps)) * K * sizeof(float), 16);
     g.off_part = static_cast<unsigned>(off);
     off = up(off + static_cast<size_t>(g.G) * 16, 16);
+    g.off_all = static_cast<unsigned>(off);
+    off = up(off + static_cast<size_t>(R) * g.G * 16, 16);
     g.off_coef = static_cast<unsigned>(off);
     off = up(off + static_cast<size_t>(g.G) * 16, 16);
     g.off_flag = static_cast<unsigned>(off);
     off = up(off + static_cast<size_t>(g.rows_max), 16);
     g.off_origin = static_cast<unsigned>(off);
-    off = up(off + static_cast<size_t>(g.rows_max) * origin_stride * sizeof(int2), 16);
+    off = up(off + std::max<size_t>(16, static_cast<size_t>(g.rows_max) * origin_stride * sizeof(int2)), 16);
     g.total_bytes = static_cast<unsigned>(off);
     return off;
 }
