@@ -162,7 +162,7 @@ struct SlabPlan {
 bool g_slab = true;            // use the one-launch path where it applies
 int g_slab_cta_kb = 112;       // preferred shared memory per block: two blocks per SM stay resident
 int g_slab_min_ctas = 0;       // grow the cluster while the launch has fewer blocks than this; 0 = 2 per SM
-int g_slab_max_mb = 1 << 20;   // tensors larger than this many MiB keep the streaming path
+int g_slab_max_mb = 6;         // tensors larger than this many MiB keep the streaming path (measured: see bns.h)
 int g_slab_cluster_max = 8;    // largest cluster (8 is the portable limit)
 constexpr size_t kSlabSmemLimit = 227 * 1024;  // most dynamic shared memory a block may ask for
 
@@ -197,21 +197,20 @@ size_t slab_layout(SlabGeom& g, int R, int tensors, int origin_stride) {
     return off;
 }
 
-// origin_stride: 0 = no device-resident patch offsets, 1 = one pair per sample, 2 = one pair per map
-SlabPlan plan_slab(int N, int C, int H, int W, int ebytes, bool backward, int offsets_kind) {
-    SlabPlan sp;
-    if (!g_slab) return sp;
+// Channel groups: the fewest channels whose row segment is a multiple of 16 bytes, doubled while the
+// segment is shorter than 512 bytes.  False if the shape does not fit the scheme (a segment wider than
+// kThreads vectors, or C not a multiple of the group).
+bool group_geometry(int N, int C, int H, int W, int ebytes, SlabGeom& g) {
     const size_t HW = static_cast<size_t>(H) * W;
-    if (H >= 32768 || W >= 65536) return sp;
-    if (static_cast<double>(N) * C * HW * ebytes > static_cast<double>(g_slab_max_mb) * 1048576.0) return sp;
+    if (H >= 32768 || W >= 65536) return false;
     const int V = 16 / ebytes;
-    int G = static_cast<int>(16 / gcd_size(HW * ebytes, 16));  // fewest channels whose row segment is a multiple of 16 bytes
-    if (C % G != 0) return sp;
+    int G = static_cast<int>(16 / gcd_size(HW * ebytes, 16));
+    if (C % G != 0) return false;
     while (static_cast<size_t>(G) * HW * ebytes < 512 && C % (2 * G) == 0 && 2 * G * HW / V <= static_cast<size_t>(kThreads) &&
-           2 * G <= 64)
+           2 * G <= kSlabMaxChannels)
         G *= 2;
-    if (G * HW / V > static_cast<size_t>(kThreads) || G > kThreads) return sp;
-    SlabGeom& g = sp.geo;
+    if (G * HW / V > static_cast<size_t>(kThreads) || G > kSlabMaxChannels) return false;
+    g = SlabGeom{};
     g.N = N;
     g.C = C;
     g.H = H;
@@ -223,6 +222,21 @@ SlabPlan plan_slab(int N, int C, int H, int W, int ebytes, bool backward, int of
     g.RL = kThreads / g.NV;
     g.P = static_cast<unsigned>(C * HW);
     g.row_bytes = static_cast<unsigned>(g.Wd * ebytes);
+    return true;
+}
+
+// Sampled elements per channel up to which a sampled set counts as small: one block can read all of it.
+int g_direct_max = 8192;
+
+// origin_stride: 0 = no device-resident patch offsets, 1 = one pair per sample, 2 = one pair per map
+SlabPlan plan_slab(int N, int C, int H, int W, int ebytes, bool backward, int offsets_kind) {
+    SlabPlan sp;
+    if (!g_slab) return sp;
+    const size_t HW = static_cast<size_t>(H) * W;
+    if (static_cast<double>(N) * C * HW * ebytes > static_cast<double>(g_slab_max_mb) * 1048576.0) return sp;
+    if (!group_geometry(N, C, H, W, ebytes, sp.geo)) return sp;
+    SlabGeom& g = sp.geo;
+    const int G = g.G;
     const int tensors = backward ? 2 : 1;
     const int stride = offsets_kind == 2 ? G : offsets_kind == 1 ? 1 : 0;
     const int groups = C / G;
@@ -260,7 +274,7 @@ struct Problem {
     ColPlan main_plan;             // all N rows of x (normalise, backward pass 1, full statistics, full backward)
     ColPlan stat_plan;             // BATCH: the k sampled rows;  VIRTUAL: the nv rows of xv
     PatchPlan patch_plan;
-    SlabPlan slab_fwd, slab_bwd;   // the one-launch path, when the layer qualifies
+    SlabPlan slab_fwd, slab_bwd;   // the one-launch on-chip path, when the layer qualifies
     // workspace layout
     size_t off_list, off_stats, off_bwd, off_bwd_v, total;
 };
@@ -418,8 +432,7 @@ bns_status clear_status(const Problem& pb, void* ws, cudaStream_t stream, unsign
 
 // ------------------------------------------------------------------------------------ launches
 bool g_pdl = true;    // ask for programmatic dependent launch (blocks may be scheduled while the previous kernel drains)
-bool g_l2_order = true;
-int g_direct_max = 8192;  // sampled elements per channel up to which one block per channel handles the sampled set  // order rows so that a kernel re-reads what the previous one left in L2
+bool g_l2_order = true;  // order rows so that a kernel re-reads what the previous one left in L2
 
 template <typename... KArgs, typename... Args>
 void launch_with(bool early_scheduling, int kind, void (*kernel)(KArgs...), unsigned grid, cudaStream_t s,
@@ -518,7 +531,7 @@ std::mutex g_slab_attr_mutex;
 template <typename... KArgs, typename... Args>
 void launch_cluster(int kind, void (*kernel)(KArgs...), unsigned grid, unsigned cluster, size_t smem, cudaStream_t s,
                     Args&&... args) {
-    {
+    if (smem > 48 * 1024) {
         static bool raised[kMaxDevices] = {};  // one array per kernel instantiation
         int device = -1;
         if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) {

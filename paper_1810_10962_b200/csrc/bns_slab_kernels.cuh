@@ -30,6 +30,7 @@ namespace bns {
 namespace cg = cooperative_groups;
 
 constexpr int kWarps = kThreads / 32;
+constexpr int kSlabMaxChannels = 64;       // most channels per cluster
 constexpr unsigned kWaitPolls = 1u << 22;  // mbarrier.try_wait attempts before a wait gives up
 
 // Waits that ran out since the library was loaded (never reset by the kernels).

@@ -12,12 +12,19 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(autouse=True, params=["onchip", "streaming"])
 def execution_path(request):
-    """Every case runs twice: with the one-launch on-chip path allowed (layers that qualify take it,
-    the others stream anyway) and with it switched off (everything streams)."""
+    """Every case runs twice: with the one-launch on-chip path taken by every layer that fits it (the size
+    limit that the library applies by default is lifted, so the mid-sized layers exercise it too; the rest
+    streams anyway), and with that path switched off (everything goes through the streaming kernels and
+    their partial sums)."""
     from paper_1810_10962_b200 import bns
     bns.set_tuning("slab", 1 if request.param == "onchip" else 0)
+    bns.set_tuning("slab_max_mb", 1 << 20)
     yield request.param
     bns.set_tuning("slab", 1)
+    bns.set_tuning("slab_max_mb", DEFAULT_SLAB_MAX_MB)
+
+
+DEFAULT_SLAB_MAX_MB = 6
 
 
 # ----------------------------------------------------------------------------- config 1: tiny
@@ -373,7 +380,7 @@ def test_every_cluster_size_matches_the_oracle(cluster_max, rule, kw, execution_
     """The combine across the blocks of a cluster, for 1 to 8 blocks; 37 samples split unevenly."""
     from paper_1810_10962_b200 import bns
     if execution_path != "onchip":
-        pytest.skip("cluster sizes only exist on the on-chip path")
+        pytest.skip("this knob belongs to the on-chip path")
     case = make_case(37, 24, 10, 10, rule, seed=91, **kw)
     try:
         bns.set_tuning("slab_cluster_max", cluster_max)
@@ -382,3 +389,19 @@ def test_every_cluster_size_matches_the_oracle(cluster_max, rule, kw, execution_
     finally:
         bns.set_tuning("slab_cluster_max", 8)
         bns.set_tuning("slab_min_ctas", 0)
+
+
+def test_default_size_limit_of_the_onchip_path():
+    """By default only tensors up to a few MiB take the on-chip path (larger ones measured faster through
+    the streaming kernels); the limit is a knob."""
+    import torch
+    from paper_1810_10962_b200 import bns
+    bns.set_tuning("slab", 1)
+    bns.set_tuning("slab_max_mb", DEFAULT_SLAB_MAX_MB)
+    sp = bns.Sampling.full()
+    small = torch.empty(128, 32, 16, 16, device="cuda")                          # 4 MiB
+    large = torch.empty(256, 256, 14, 14, device="cuda", dtype=torch.bfloat16)   # 24.5 MiB
+    assert bns.slab_plan(small, sp) is not None and bns.slab_plan(small, sp, backward=True) is not None
+    assert bns.slab_plan(large, sp) is None
+    bns.set_tuning("slab_max_mb", 64)
+    assert bns.slab_plan(large, sp) is not None
