@@ -362,7 +362,10 @@ const char* bns_kernel_name(int kernel_kind);
  * partial sums, 0 = never; "nhwc_blocks": blocks per launch of the channels-last kernels (each block leaves one partial per
  * channel); "slab": 0/1 use the one-launch path where it applies, "slab_cta_kb": preferred shared memory per block of
  * that path in KiB, "slab_min_ctas": grow its clusters while a launch has fewer blocks (0 = two per SM), "slab_max_mb":
- * tensors above this many MiB keep the streaming path, "slab_cluster_max": largest cluster (1..8);
+ * tensors above this many MiB keep the streaming path (default 6: measured on B200, larger tensors run faster through
+ * the streaming kernels), "slab_small_sets": 0/1 take that path also when the sampled set is small (default 0: the
+ * streaming path is then two short kernels per direction and measured faster), "slab_cluster_max": largest cluster (1..8);
+ * "per_channel_min_hw": map size H*W from which backward pass 1 keeps its sums per channel instead of per position;
  * "pdl": 0/1 programmatic dependent launch; "l2_order": 0/1 visit rows in an
  * order that lets a kernel find in L2 what the previous one read.  Returns BNS_OK,
  * BNS_ERR_RULE for an unknown name or BNS_ERR_SHAPE for a value < 1. */

@@ -164,6 +164,7 @@ int g_slab_cta_kb = 112;       // preferred shared memory per block: two blocks 
 int g_slab_min_ctas = 0;       // grow the cluster while the launch has fewer blocks than this; 0 = 2 per SM
 int g_slab_max_mb = 6;         // tensors larger than this many MiB keep the streaming path (measured: see bns.h)
 int g_slab_cluster_max = 8;    // largest cluster (8 is the portable limit)
+bool g_slab_small_sets = false;  // also for small sampled sets (whose streaming path is short already; measured slower)
 constexpr size_t kSlabSmemLimit = 227 * 1024;  // most dynamic shared memory a block may ask for
 
 size_t gcd_size(size_t a, size_t b) { return b ? gcd_size(b, a % b) : a; }
@@ -377,8 +378,10 @@ bns_status make_problem(const bns_shape* sh, const bns_sampling* sp, Problem& pb
     if (sp->rule == BNS_RULE_VIRTUAL) off += align_up(pb.stat_plan.partial_count() * sizeof(float2));
     pb.total = off;
     const int offsets_kind = (sp->rule == BNS_RULE_FEATURE && pb.patch.offsets) ? (pb.patch.stride_c ? 2 : 1) : 0;
-    pb.slab_fwd = plan_slab(pb.N, pb.C, pb.H, pb.W, eb, false, offsets_kind);
-    pb.slab_bwd = plan_slab(pb.N, pb.C, pb.H, pb.W, eb, true, offsets_kind);
+    if (g_slab_small_sets || sp->rule == BNS_RULE_FULL || pb.s > static_cast<double>(g_direct_max)) {
+        pb.slab_fwd = plan_slab(pb.N, pb.C, pb.H, pb.W, eb, false, offsets_kind);
+        pb.slab_bwd = plan_slab(pb.N, pb.C, pb.H, pb.W, eb, true, offsets_kind);
+    }
     return BNS_OK;
 }
 
@@ -502,6 +505,18 @@ const typename T::storage* in(const void* p) {
 template <typename T>
 typename T::storage* out(void* p) {
     return static_cast<typename T::storage*>(p);
+}
+
+// Backward pass 1 keeps its sums per channel where the maps are large and per position where they are
+// small (see col_bwd_reduce_kernel); one element per thread always takes the per-position form.
+int g_per_channel_min_hw = 512;
+
+template <typename T, int V, bool WRITE_DX>
+auto bwd_reduce_variant(int HW) -> decltype(&col_bwd_reduce_kernel<T, V, WRITE_DX, false>) {
+    if constexpr (V >= 2) {
+        if (HW >= V && HW >= g_per_channel_min_hw) return col_bwd_reduce_kernel<T, V, WRITE_DX, true>;
+    }
+    return col_bwd_reduce_kernel<T, V, WRITE_DX, false>;
 }
 
 unsigned warp_per_channel_grid(int C) { return static_cast<unsigned>((C + kThreads / 32 - 1) / (kThreads / 32)); }
@@ -705,17 +720,17 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
         order = RowOrder{RowOrder::kRangeLast, pb.N, pb.begin, pb.count};
     if (full)
         BNS_BY_TYPE_V(pb.dtype, pl.V,
-                      (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, false>, pl.grid(), stream, in<T>(x),
+                      (launch(BNS_KERNEL_BWD_REDUCE, bwd_reduce_variant<T, V, false>(pb.HW), pl.grid(), stream, in<T>(x),
                               in<T>(dy), out<T>(nullptr), gamma, mean, invstd, order, pl.nchunks, pl.tiles, pb.HW, pb.P,
                               false, sink)));
     else
         BNS_BY_TYPE_V(pb.dtype, pl.V,
-                      (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, true>, pl.grid(), stream, in<T>(x),
+                      (launch(BNS_KERNEL_BWD_REDUCE, bwd_reduce_variant<T, V, true>(pb.HW), pl.grid(), stream, in<T>(x),
                               in<T>(dy), out<T>(dx), gamma, mean, invstd, order, pl.nchunks, pl.tiles, pb.HW, pb.P, false,
                               sink)));
     if (virtual_grads)
         BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
-                      (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, false>, pv.grid(), stream, in<T>(sp->xv),
+                      (launch(BNS_KERNEL_BWD_REDUCE, bwd_reduce_variant<T, V, false>(pb.HW), pv.grid(), stream, in<T>(sp->xv),
                               in<T>(sp->dyv), out<T>(nullptr), gamma, mean, invstd,
                               RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P, true,
                               sink)));
@@ -851,12 +866,12 @@ bns_status backward_mixed_impl(const MixedProblem& mp, const bns_sampling* sp, c
                   pq.layout(), invstd, dgamma, dbeta};
     // the sums of Eq. 5 over the real batch (and dx without the statistics terms), then over the virtual rows
     BNS_BY_TYPE_V(pr.dtype, pl.V,
-                  (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, true>, pl.grid(), stream, in<T>(x), in<T>(dy),
+                  (launch(BNS_KERNEL_BWD_REDUCE, bwd_reduce_variant<T, V, true>(pr.HW), pl.grid(), stream, in<T>(x), in<T>(dy),
                           out<T>(dx), gamma, mean, invstd, RowOrder{RowOrder::kIdentity, pr.N, 0, 0}, pl.nchunks, pl.tiles,
                           pr.HW, pr.P, false, sink)));
     if (sp->dyv)
         BNS_BY_TYPE_V(sp->xv_dtype, pq.V,
-                      (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, false>, pq.grid(), stream, in<T>(sp->xv),
+                      (launch(BNS_KERNEL_BWD_REDUCE, bwd_reduce_variant<T, V, false>(pr.HW), pq.grid(), stream, in<T>(sp->xv),
                               in<T>(sp->dyv), out<T>(nullptr), gamma, mean, invstd,
                               RowOrder{RowOrder::kIdentity, pq.rows, 0, 0}, pq.nchunks, pq.tiles, pr.HW, pr.P, true,
                               sink)));
@@ -1338,10 +1353,12 @@ int bns_set_tuning(const char* name, int value) {
                  {"direct_max", &g_direct_max, nullptr, true},
                  {"nhwc_blocks", &g_nhwc_blocks, nullptr, true},
                  {"slab", nullptr, &g_slab, false},
+                 {"slab_small_sets", nullptr, &g_slab_small_sets, false},
                  {"slab_cta_kb", &g_slab_cta_kb, nullptr, false},
                  {"slab_min_ctas", &g_slab_min_ctas, nullptr, true},
                  {"slab_max_mb", &g_slab_max_mb, nullptr, false},
                  {"slab_cluster_max", &g_slab_cluster_max, nullptr, false},
+                 {"per_channel_min_hw", &g_per_channel_min_hw, nullptr, false},
                  {"pdl", nullptr, &g_pdl, false},
                  {"l2_order", nullptr, &g_l2_order, false}};
     for (const Knob& k : knobs) {
@@ -1534,7 +1551,7 @@ bns_status bns_sync_backward_sums(const bns_shape* shape, const void* x, const v
     // row 0: sum dy (dbeta), row 1: sum dy xhat (dgamma) over this rank's elements
     GradSink sink{ws_at<float2>(workspace, pb.off_bwd), pl.layout(), nullptr, pl.layout(), invstd, sums + pb.C, sums};
     BNS_BY_TYPE_V(pb.dtype, pl.V,
-                  (launch(BNS_KERNEL_BWD_REDUCE, col_bwd_reduce_kernel<T, V, true>, pl.grid(), stream, in<T>(x), in<T>(dy),
+                  (launch(BNS_KERNEL_BWD_REDUCE, bwd_reduce_variant<T, V, true>(pb.HW), pl.grid(), stream, in<T>(x), in<T>(dy),
                           out<T>(dx), gamma, mean, invstd, RowOrder{RowOrder::kIdentity, pb.N, 0, 0}, pl.nchunks, pl.tiles,
                           pb.HW, pb.P, false, sink)));
     launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);

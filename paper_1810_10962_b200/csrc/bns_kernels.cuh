@@ -141,6 +141,56 @@ struct Vec {
     }
 };
 
+// Two fp32 values in one 64-bit register pair, for the packed fp32x2 arithmetic of sm_100 (each half is
+// an ordinary round-to-nearest fp32 operation, so results equal the scalar ones bit for bit).
+using pair_t = unsigned long long;
+__device__ __forceinline__ pair_t make_pair(float lo, float hi) {
+    pair_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void split_pair(pair_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ pair_t add2(pair_t a, pair_t b) {
+    pair_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ pair_t mul2(pair_t a, pair_t b) {
+    pair_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ pair_t fma2(pair_t a, pair_t b, pair_t c) {
+    pair_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+// Elements 2q and 2q+1 of a vector as a pair, and back (bf16: one 32-bit word holds both).
+template <typename T, int V>
+__device__ __forceinline__ pair_t vec_pair(const Vec<T, V>& v, int q) {
+    if constexpr (sizeof(typename T::storage) == 2) {
+        const unsigned w = reinterpret_cast<const unsigned*>(&v.raw)[q];
+        return make_pair(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+    } else {
+        const float* f = reinterpret_cast<const float*>(&v.raw);
+        return make_pair(f[2 * q], f[2 * q + 1]);
+    }
+}
+template <typename T, int V>
+__device__ __forceinline__ void set_vec_pair(Vec<T, V>& v, int q, pair_t p) {
+    float lo, hi;
+    split_pair(p, lo, hi);
+    if constexpr (sizeof(typename T::storage) == 2) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);  // low half = first argument
+        reinterpret_cast<unsigned*>(&v.raw)[q] = *reinterpret_cast<unsigned*>(&h);
+    } else {
+        float* f = reinterpret_cast<float*>(&v.raw);
+        f[2 * q] = lo;
+        f[2 * q + 1] = hi;
+    }
+}
+
 // Channels of the V positions p .. p+V-1 (HW may be smaller than V).
 template <int V>
 __device__ __forceinline__ void position_channels(unsigned p, int HW, int (&c)[V]) {
@@ -656,100 +706,216 @@ col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::stor
 }
 
 // ------------------------------------------------------------------------------------ backward, pass 1
+// Folds per-THREAD sums into one (sum dy, sum dy (x - mean)) pair per channel the tile meets, for tiles
+// whose threads hold V consecutive positions of maps at least V positions large: a thread then meets at
+// most two channels, c0 (its first position's) and, if its positions straddle a map boundary, c0 + 1.
+// s_first[t] holds thread t's sums over its positions in c0, s_second[t] those in c0 + 1 (zero unless it
+// straddles).  The threads of a channel are consecutive, so a slot's total is the sum of s_first over a
+// range of threads plus s_second of the one thread just before that range when it straddles into it.
+template <int V>
+__device__ __forceinline__ void fold_thread_sums(const float2* s_first, const float2* s_second, const TileChannels& tc,
+                                                 int HW, float2* out) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int slot = warp; slot < tc.nslots; slot += kThreads / 32) {
+        unsigned lo, hi;  // positions of the slot's channel inside the tile, relative to its first position
+        tc.range(slot, HW, lo, hi);
+        const int t_lo = static_cast<int>((lo + V - 1) / V);  // first thread whose first position lies in the channel
+        const int t_hi = static_cast<int>((hi + V - 1) / V);
+        float sa = 0.f, sb = 0.f;
+        for (int t = t_lo + lane; t < t_hi; t += 32) {
+            const float2 v = s_first[t];
+            sa += v.x;
+            sb += v.y;
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            sa += __shfl_down_sync(0xffffffffu, sa, d);
+            sb += __shfl_down_sync(0xffffffffu, sb, d);
+        }
+        if (lane == 0) {
+            if (lo % V != 0) {  // the thread before t_lo starts in the previous channel and ends in this one
+                const float2 v = s_second[t_lo - 1];
+                sa += v.x;
+                sb += v.y;
+            }
+            out[slot] = make_float2(sa, sb);
+        }
+    }
+}
+
 // Streams dy and x once: per channel partial sums of dy and dy (x - mean) and, if WRITE_DX, the
 // gradient of every element without the statistics terms, dx = gamma invstd dy (lower branch of Eq. 6).
-template <typename T, int V, bool WRITE_DX>
-__global__ void __launch_bounds__(kThreads)
+// PER_CHANNEL selects how a thread keeps its sums when every map holds at least V positions: per channel
+// (few registers, four blocks per SM even for bf16; pays extra arithmetic in every warp that holds a
+// thread straddling two maps - right for large maps, where such threads are rare) or per position (no
+// special case for straddling threads - right for small maps, where most warps hold one).
+template <typename T, int V, bool WRITE_DX, bool PER_CHANNEL>
+__global__ void __launch_bounds__(kThreads, PER_CHANNEL ? 4 : 3)
 col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
                       typename T::storage* __restrict__ dx, const float* __restrict__ gamma,
                       const float* __restrict__ mean, const float* __restrict__ invstd, RowOrder order, int nchunks,
                       unsigned tiles, int HW, unsigned P, bool virtual_pass, GradSink G) {
     constexpr unsigned TP = kThreads * V;
-    __shared__ float s_dy[TP];
-    __shared__ float s_dyxc[TP];
+    // per-position sums (maps smaller than a vector) or, reusing the space, per-thread sums
+    __shared__ __align__(16) float s_sums[2 * TP];
     grid_dependency_wait();
     grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
     const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
-    float acc_dy[V], acc_dyxc[V];
-#pragma unroll
-    for (int j = 0; j < V; ++j) acc_dy[j] = acc_dyxc[j] = 0.f;
-    if (p < P) {
-        float a[V], mu[V];
-        if (HW >= V) {  // at most two channels per thread: two parameter sets, selected per position
+    float2* out = (virtual_pass ? G.partials_v : G.partials) +
+                  (static_cast<size_t>(ck) * tiles + tile) * (virtual_pass ? G.Lv.max_slots : G.L.max_slots);
+    const typename T::storage* xp = x + p;
+    const typename T::storage* gp = dy + p;
+    typename T::storage* op = WRITE_DX ? dx + p : nullptr;
+    if (PER_CHANNEL) {
+        // Sums of g and of g (x - pivot) with the pivot the mean of the thread's first channel (one register
+        // instead of a mean per position); the deviation from each channel's own mean is put right after the
+        // loop: sum g (x - mean) = sum g (x - pivot) - (mean - pivot) sum g.
+        // Every thread sums over all its V positions with packed fp32x2 arithmetic (one packed accumulator
+        // per sum).  The rare thread whose positions straddle two channels also sums the second channel's
+        // share on the side, element by element, inside the same loop - the loads are shared, so a warp that
+        // holds such a thread only executes some more arithmetic.
+        constexpr int Q = V >= 2 ? V / 2 : 1;
+        float2* s_first = reinterpret_cast<float2*>(s_sums);
+        float2* s_second = s_first + kThreads;
+        float2 first = make_float2(0.f, 0.f), second = make_float2(0.f, 0.f);
+        if (p < P) {
             const TwoChannels ch(p, HW, V);
+            const bool straddle = ch.jb < V;
             const float mu0 = mean[ch.c0], mu1 = mean[ch.c1];
             const float a0 = WRITE_DX ? gamma[ch.c0] * invstd[ch.c0] : 0.f;
             const float a1 = WRITE_DX ? gamma[ch.c1] * invstd[ch.c1] : 0.f;
+            const pair_t minus_pivot = make_pair(-mu0, -mu0);
+            const pair_t a2 = make_pair(a0, a0);
+            pair_t sum_g = make_pair(0.f, 0.f), sum_gx = make_pair(0.f, 0.f);
+            float s1_g = 0.f, s1_gx = 0.f;  // share of channel c1 (positions j >= jb)
+            // batches of kUnroll rows, all loads of a batch in flight together; the last batch may be short
+            for (int i = ck; i < order.rows; i += kUnroll * nchunks) {
+                Vec<T, V> vx[kUnroll], vg[kUnroll];
+                int row[kUnroll];
 #pragma unroll
-            for (int j = 0; j < V; ++j) {
-                mu[j] = ch.pick(j, mu0, mu1);
-                a[j] = ch.pick(j, a0, a1);
-            }
-        } else {
-            int c[V];
-            position_channels<V>(p, HW, c);
+                for (int u = 0; u < kUnroll; ++u) {
+                    if (i + u * nchunks < order.rows) {
+                        row[u] = order(i + u * nchunks);
+                        vx[u].load(xp + static_cast<size_t>(row[u]) * P);
+                        vg[u].load(gp + static_cast<size_t>(row[u]) * P);
+                    }
+                }
 #pragma unroll
-            for (int j = 0; j < V; ++j) {
-                mu[j] = mean[c[j]];
-                a[j] = WRITE_DX ? gamma[c[j]] * invstd[c[j]] : 0.f;
+                for (int u = 0; u < kUnroll; ++u) {
+                    if (i + u * nchunks < order.rows) {
+                        pair_t g2[Q];
+#pragma unroll
+                        for (int q = 0; q < Q; ++q) {
+                            g2[q] = vec_pair<T, V>(vg[u], q);
+                            sum_gx = fma2(g2[q], add2(vec_pair<T, V>(vx[u], q), minus_pivot), sum_gx);
+                        }
+                        if (straddle) {
+#pragma unroll
+                            for (int q = 0; q < Q; ++q) {
+                                float g[2];
+                                split_pair(g2[q], g[0], g[1]);
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    const bool in_second = 2 * q + h >= ch.jb;
+                                    s1_g += in_second ? g[h] : 0.f;
+                                    s1_gx = fmaf(in_second ? g[h] : 0.f, vx[u].get(2 * q + h) - mu0, s1_gx);
+                                    if (WRITE_DX) g[h] *= in_second ? a1 : a0;
+                                }
+                                if (WRITE_DX) set_vec_pair<T, V>(vg[u], q, make_pair(g[0], g[1]));
+                            }
+                        } else if (WRITE_DX) {
+#pragma unroll
+                            for (int q = 0; q < Q; ++q) set_vec_pair<T, V>(vg[u], q, mul2(g2[q], a2));
+                        }
+                        if (WRITE_DX) vg[u].store(op + static_cast<size_t>(row[u]) * P);
+#pragma unroll
+                        for (int w = Q / 2; w > 0; w >>= 1)
+#pragma unroll
+                            for (int q = 0; q < w; ++q) g2[q] = add2(g2[q], g2[q + w]);
+                        sum_g = add2(sum_g, g2[0]);
+                    }
+                }
             }
+            float lo, hi;
+            split_pair(sum_g, lo, hi);
+            first.x = lo + hi - s1_g;
+            split_pair(sum_gx, lo, hi);
+            first.y = lo + hi - s1_gx;
+            second = make_float2(s1_g, fmaf(-(mu1 - mu0), s1_g, s1_gx));
         }
-        const typename T::storage* xp = x + p;
-        const typename T::storage* gp = dy + p;
-        typename T::storage* op = WRITE_DX ? dx + p : nullptr;
-        int i = ck;
-        for (; i + (kUnroll - 1) * nchunks < order.rows; i += kUnroll * nchunks) {
-            Vec<T, V> vx[kUnroll], vg[kUnroll];
-            int row[kUnroll];
+        s_first[threadIdx.x] = first;
+        s_second[threadIdx.x] = second;
+        __syncthreads();
+        fold_thread_sums<V>(s_first, s_second, TileChannels(tile, TP, P, HW), HW, out);
+    } else {
+        // a mean and a pair of sums per position
+        float* s_dy = s_sums;
+        float* s_dyxc = s_sums + TP;
+        float acc_dy[V], acc_dyxc[V];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                row[u] = order(i + u * nchunks);
-                vx[u].load(xp + static_cast<size_t>(row[u]) * P);
-                vg[u].load(gp + static_cast<size_t>(row[u]) * P);
-            }
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                float g[V], xv[V];
-                vg[u].unpack(g);
-                vx[u].unpack(xv);
+        for (int j = 0; j < V; ++j) acc_dy[j] = acc_dyxc[j] = 0.f;
+        if (p < P) {
+            float a[V], mu[V];
+            if (HW >= V) {  // at most two channels per thread: two parameter sets, selected per position
+                const TwoChannels ch(p, HW, V);
+                const float mu0 = mean[ch.c0], mu1 = mean[ch.c1];
+                const float a0 = WRITE_DX ? gamma[ch.c0] * invstd[ch.c0] : 0.f;
+                const float a1 = WRITE_DX ? gamma[ch.c1] * invstd[ch.c1] : 0.f;
 #pragma unroll
                 for (int j = 0; j < V; ++j) {
-                    acc_dy[j] += g[j];
-                    acc_dyxc[j] = fmaf(g[j], xv[j] - mu[j], acc_dyxc[j]);
-                    if (WRITE_DX) g[j] *= a[j];
+                    mu[j] = ch.pick(j, mu0, mu1);
+                    a[j] = ch.pick(j, a0, a1);
                 }
-                if (WRITE_DX) {
-                    vg[u].pack(g);
-                    vg[u].store(op + static_cast<size_t>(row[u]) * P);
+            } else {
+                int c[V];
+                position_channels<V>(p, HW, c);
+#pragma unroll
+                for (int j = 0; j < V; ++j) {
+                    mu[j] = mean[c[j]];
+                    a[j] = WRITE_DX ? gamma[c[j]] * invstd[c[j]] : 0.f;
+                }
+            }
+            for (int i = ck; i < order.rows; i += kUnroll * nchunks) {
+                Vec<T, V> vx[kUnroll], vg[kUnroll];
+                int row[kUnroll];
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    if (i + u * nchunks < order.rows) {
+                        row[u] = order(i + u * nchunks);
+                        vx[u].load(xp + static_cast<size_t>(row[u]) * P);
+                        vg[u].load(gp + static_cast<size_t>(row[u]) * P);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    if (i + u * nchunks < order.rows) {
+                        float g[V], xv[V];
+                        vg[u].unpack(g);
+                        vx[u].unpack(xv);
+#pragma unroll
+                        for (int j = 0; j < V; ++j) {
+                            acc_dy[j] += g[j];
+                            acc_dyxc[j] = fmaf(g[j], xv[j] - mu[j], acc_dyxc[j]);
+                            if (WRITE_DX) g[j] *= a[j];
+                        }
+                        if (WRITE_DX) {
+                            vg[u].pack(g);
+                            vg[u].store(op + static_cast<size_t>(row[u]) * P);
+                        }
+                    }
                 }
             }
         }
-        for (; i < order.rows; i += nchunks) {
-            const size_t off = static_cast<size_t>(order(i)) * P;
-            Vec<T, V> vx, vg;
-            vx.load(xp + off);
-            vg.load(gp + off);
 #pragma unroll
-            for (int j = 0; j < V; ++j) {
-                float g = vg.get(j);
-                acc_dy[j] += g;
-                acc_dyxc[j] = fmaf(g, vx.get(j) - mu[j], acc_dyxc[j]);
-                if (WRITE_DX) vg.set(j, a[j] * g);
-            }
-            if (WRITE_DX) vg.store(op + off);
+        for (int j = 0; j < V; ++j) {
+            s_dy[threadIdx.x * V + j] = acc_dy[j];
+            s_dyxc[threadIdx.x * V + j] = acc_dyxc[j];
         }
+        __syncthreads();
+        fold_sums(s_dy, s_dyxc, TileChannels(tile, TP, P, HW), HW, out);
     }
-#pragma unroll
-    for (int j = 0; j < V; ++j) {
-        s_dy[threadIdx.x * V + j] = acc_dy[j];
-        s_dyxc[threadIdx.x * V + j] = acc_dyxc[j];
-    }
-    __syncthreads();
-    float2* out = (virtual_pass ? G.partials_v : G.partials) +
-                  (static_cast<size_t>(ck) * tiles + tile) * (virtual_pass ? G.Lv.max_slots : G.L.max_slots);
-    fold_sums(s_dy, s_dyxc, TileChannels(tile, TP, P, HW), HW, out);
 }
 
 // ------------------------------------------------------------------------------------ backward, statistics terms

@@ -12,16 +12,18 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(autouse=True, params=["onchip", "streaming"])
 def execution_path(request):
-    """Every case runs twice: with the one-launch on-chip path taken by every layer that fits it (the size
-    limit that the library applies by default is lifted, so the mid-sized layers exercise it too; the rest
-    streams anyway), and with that path switched off (everything goes through the streaming kernels and
-    their partial sums)."""
+    """Every case runs twice: with the one-launch on-chip path taken by every layer that fits it (the limits
+    that the library applies by default - small tensors only, not for small sampled sets - are lifted, so
+    the mid-sized layers and every rule exercise it too; the rest streams anyway), and with that path
+    switched off (everything goes through the streaming kernels and their partial sums)."""
     from paper_1810_10962_b200 import bns
     bns.set_tuning("slab", 1 if request.param == "onchip" else 0)
     bns.set_tuning("slab_max_mb", 1 << 20)
+    bns.set_tuning("slab_small_sets", 1)
     yield request.param
     bns.set_tuning("slab", 1)
     bns.set_tuning("slab_max_mb", DEFAULT_SLAB_MAX_MB)
+    bns.set_tuning("slab_small_sets", 0)
 
 
 DEFAULT_SLAB_MAX_MB = 6
@@ -398,6 +400,7 @@ def test_default_size_limit_of_the_onchip_path():
     from paper_1810_10962_b200 import bns
     bns.set_tuning("slab", 1)
     bns.set_tuning("slab_max_mb", DEFAULT_SLAB_MAX_MB)
+    bns.set_tuning("slab_small_sets", 0)
     sp = bns.Sampling.full()
     small = torch.empty(128, 32, 16, 16, device="cuda")                          # 4 MiB
     large = torch.empty(256, 256, 14, 14, device="cuda", dtype=torch.bfloat16)   # 24.5 MiB
@@ -405,3 +408,8 @@ def test_default_size_limit_of_the_onchip_path():
     assert bns.slab_plan(large, sp) is None
     bns.set_tuning("slab_max_mb", 64)
     assert bns.slab_plan(large, sp) is not None
+    # small sampled sets keep their short streaming path unless asked otherwise
+    few = bns.Sampling.feature(4, 4, np.array([0, 0]))
+    assert bns.slab_plan(small, few) is None
+    bns.set_tuning("slab_small_sets", 1)
+    assert bns.slab_plan(small, few) is not None
