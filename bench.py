@@ -3,7 +3,10 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
-A *step* is one forward+backward of every layer of the workload through the C ABI.  The default
+A *step* is one forward+backward of every layer of the workload through the C ABI.  The K steps of
+``--steps`` are timed as one loop between two CUDA events; that loop is repeated (at least 30 times and for
+at least ``--seconds``) and the reported time per step is the median over the repetitions, with the
+minimum beside it.  The default
 workload is the ImageNet ResNet-18 stage-1 layer, fp32 (256,64,56,56), once with Batch Sampling
 (k = 32 of 256) and once with Feature Sampling (8x8 patch), and the same layer through the library's
 full BN for the speed-up figure.  The metric is algorithmic GB/s: the bytes the method itself must
@@ -37,10 +40,10 @@ import bns_inputs as I  # noqa: E402
 EPS = 1e-5
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one col_bwd_reduce_kernel<F32,4,true> launch on the default
-# workload's layer shape (256x64x56x56 fp32), from the ncu capture summarised in
-# profiles/col_bwd_reduce_f32_resnet18_stage1.md; reported only for that workload.
-BWD_REDUCE_DRAM_TRAFFIC_BYTES = 580_750_336   # 411.14 MB read + 169.61 MB written (rest of dx still dirty in L2)
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of backward pass 1 (fp32, 16-byte vectors, writing dx)
+# on the default workload's layer shape (256x64x56x56 fp32), from an ncu capture of this very kernel; reported
+# only for that workload.  None whenever the kernel has changed since the counters were taken.
+BWD_REDUCE_DRAM_TRAFFIC_BYTES = None
 
 
 # ----------------------------------------------------------------------------- workloads
@@ -161,6 +164,40 @@ def host_inputs(layer: Layer, seed):
     return dict(x=x, dy=dy, gamma=gamma, beta=beta, **extra)
 
 
+def device_inputs(layer: Layer, seed, torch):
+    """The same recipe as host_inputs, drawn on the device (torch's generator instead of the host one): used for
+    the secondary workloads, whose inputs no CPU code reads.  3x3 box blur (replicated border) of N(0,1) noise
+    plus a per-channel offset U(-1,1); dy, residual and virtual samples N(0,1); gamma U(0.5,1.5); beta N(0, 0.1)."""
+    import torch.nn.functional as F
+    N, C, H, W = layer.N, layer.C, layer.H, layer.W
+    dt = torch.float32 if layer.dtype == "f32" else torch.bfloat16
+    g = torch.Generator(device="cuda")
+    g.manual_seed(int(seed))
+    offset = torch.rand(C, generator=g, device="cuda") * 2.0 - 1.0
+    x = torch.empty(N, C, H, W, device="cuda", dtype=dt)
+    block = max(1, (1 << 26) // max(1, C * H * W))           # sample blocks keep the fp32 temporaries small
+    for n0 in range(0, N, block):
+        n1 = min(N, n0 + block)
+        noise = torch.randn(n1 - n0, C, H, W, generator=g, device="cuda")
+        blurred = F.avg_pool2d(F.pad(noise, (1, 1, 1, 1), mode="replicate"), 3, stride=1)
+        x[n0:n1] = (blurred + offset[None, :, None, None]).to(dt)
+    dy = torch.empty(N, C, H, W, device="cuda", dtype=dt)
+    for n0 in range(0, N, block):
+        n1 = min(N, n0 + block)
+        dy[n0:n1] = torch.randn(n1 - n0, C, H, W, generator=g, device="cuda").to(dt)
+    out = dict(x=x, dy=dy, gamma=torch.rand(C, generator=g, device="cuda") + 0.5,
+               beta=torch.randn(C, generator=g, device="cuda") * 0.1)
+    if layer.rule == "batch":
+        out["sample_idx"] = I.batch_sample_indices(N, layer.kw["k"], seed, contiguous=True)
+    if layer.rule in ("feature", "mixed", "relu"):
+        out["offsets"] = I.patch_offsets(N, C, H, W, layer.kw["ph"], layer.kw["pw"], I.OFFSETS_SHARED, seed)
+    if layer.rule in ("virtual", "mixed"):
+        out["xv"] = torch.randn(layer.kw["nv"], C, H, W, generator=g, device="cuda")
+    if layer.rule == "relu":
+        out["residual"] = torch.randn(N, C, H, W, generator=g, device="cuda").to(dt)
+    return out
+
+
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
@@ -168,7 +205,7 @@ class ClockSampler(threading.Thread):
                0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
     REJECT = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
 
-    def __init__(self, index, period=0.005):
+    def __init__(self, index, period=0.002):
         super().__init__(daemon=True)
         self.index, self.period = index, period
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -235,14 +272,17 @@ class DeviceLayer:
         dt = torch.float32 if layer.dtype == "f32" else torch.bfloat16
 
         def dev(a):
-            t = torch.from_numpy(a).cuda().to(dt)           # exact: the values are representable in dt
+            t = a if torch.is_tensor(a) else torch.from_numpy(a).cuda().to(dt)   # exact: the values are representable in dt
             return t.permute(0, 2, 3, 1).contiguous() if nhwc else t
+
+        def vec(a):
+            return a if torch.is_tensor(a) else torch.from_numpy(a).cuda()
 
         x, dy = dev(host["x"]), dev(host["dy"])
         self.sets = [(x, dy, torch.empty_like(x), torch.empty_like(x))]
         for _ in range(sets - 1):
             self.sets.append((x.clone(), dy.clone(), torch.empty_like(x), torch.empty_like(x)))
-        self.gamma, self.beta = torch.from_numpy(host["gamma"]).cuda(), torch.from_numpy(host["beta"]).cuda()
+        self.gamma, self.beta = vec(host["gamma"]), vec(host["beta"])
         C = layer.C
         self.mean, self.invstd, self.dgamma, self.dbeta = (torch.empty(C, device="cuda") for _ in range(4))
         if nhwc:
@@ -269,14 +309,14 @@ class DeviceLayer:
         elif layer.rule == "feature":
             self.sp = bns.Sampling.feature(layer.kw["ph"], layer.kw["pw"], host["offsets"])
         elif layer.rule == "mixed":
-            xv = torch.from_numpy(host["xv"]).cuda()
+            xv = vec(host["xv"])
             self.sp = bns.Sampling.feature(layer.kw["ph"], layer.kw["pw"], host["offsets"]).with_virtual(
                 xv, yv=torch.empty_like(xv), dyv=None, dxv=torch.empty_like(xv))
             self.mean_s, self.mean_v = (torch.empty(C, device="cuda") for _ in range(2))
             self.ws = torch.empty(bns.workspace_bytes_mixed(x, self.sp), dtype=torch.uint8, device="cuda")
             return
         else:
-            xv = torch.from_numpy(host["xv"]).cuda()
+            xv = vec(host["xv"])
             self.sp = bns.Sampling.virtual(xv, yv=torch.empty_like(xv), dyv=None, dxv=torch.empty_like(xv))
         self.ws = bns.new_workspace(x, self.sp)
         # argument marshalling done once per buffer set; a step is then two C calls per layer
@@ -372,33 +412,140 @@ def whole_job_gbps(step_bytes, world, ms):
     return world * step_bytes / (ms * 1e-3) / 1e9
 
 
-def time_steps(torch, dist, run_step, steps, warmup, device_index, world):
-    """W warm-up steps, then exactly K steps between CUDA events on the current stream, bracketed by a
-    barrier and a device synchronise on both sides.  Returns (ms per step: max over ranks, clocks)."""
+def time_steps(torch, dist, run_step, steps, warmup, device_index, world, min_repeats=1, min_seconds=0.0):
+    """W warm-up steps, then R repetitions of exactly K steps, each repetition between its own pair of CUDA
+    events on the current stream, the whole timed region bracketed by a barrier and a device synchronise on
+    both sides.  R is at least `min_repeats` and large enough for the region to last `min_seconds`.
+    Returns (median ms per step: max over ranks, clocks, statistics of the repetitions)."""
     begin = getattr(run_step, "begin", lambda n: None)
     begin(warmup)
     for i in range(warmup):
         run_step(i)
     torch.cuda.synchronize()
+    repeats = max(1, min_repeats)
+    if min_seconds > 0:
+        # one untimed repetition to size the region
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        begin(steps)
+        a.record()
+        for i in range(steps):
+            run_step(warmup + i)
+        b.record()
+        torch.cuda.synchronize()
+        repeats = max(repeats, int(np.ceil(min_seconds * 1e3 / max(1e-3, a.elapsed_time(b)))))
+        repeats = min(repeats, 2000)
     if world > 1:
+        r = torch.tensor([repeats], device="cuda", dtype=torch.int64)
+        dist.all_reduce(r, op=dist.ReduceOp.MAX)
+        repeats = int(r.item())
         dist.barrier()
     torch.cuda.synchronize()
     sampler = ClockSampler(device_index)
     sampler.start()
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    begin(steps)
-    start.record()
-    for i in range(steps):
-        run_step(warmup + i)
-    stop.record()
+    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(repeats)]
+    for start, stop in events:
+        begin(steps)
+        start.record()
+        for i in range(steps):
+            run_step(warmup + i)
+        stop.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
-    ms = start.elapsed_time(stop) / steps
+    per_step = np.array([start.elapsed_time(stop) / steps for start, stop in events])
+    ms = float(np.median(per_step))
+    stats = {"repeats": repeats, "steps_per_repeat": steps, "median_ms": round(ms, 5), "min_ms": round(float(per_step.min()), 5),
+             "max_ms": round(float(per_step.max()), 5), "timed_region_ms": round(float(per_step.sum() * steps), 2)}
     if world > 1:
         ms = slowest_rank_ms(torch, dist, ms, world, "cuda")
         dist.barrier()
     torch.cuda.synchronize()
-    return ms, clocks
+    return ms, clocks, stats
+
+
+def full_bn_bytes(layers):
+    """Full BN: 3 passes forward + 5 backward; with the fused residual + ReLU 4 + 9 (residual read three times,
+    dresidual written, the second backward pass re-reads x, residual and dy)."""
+    return sum(l.count * ((13 if l.rule == "relu" else 8) * l.elems * l.ebytes + 32 * l.C) for l in layers)
+
+
+def buffer_sets(layers):
+    """Rotating buffer sets, so that no tensor is reused before more than 2x L2 (126 MB) of other data went by."""
+    bytes_per_tensor_set = sum(4 * l.elems * l.ebytes for l in layers)
+    return 2 if bytes_per_tensor_set >= 512e6 else min(8, max(2, int(np.ceil(512e6 / bytes_per_tensor_set))))
+
+
+def measure_workload(torch, dist, bns, args, layers, inputs, local, world, seconds, layer_seconds, per_layer=True,
+                     warm=True, dev=None):
+    """Times one workload: the whole step (sampled), the same layers through full BN, and each layer alone;
+    every number is the median over at least 30 repetitions of `--steps` steps.  Returns (dict, device layers)."""
+    nhwc = args.layout == "nhwc"
+    sets = buffer_sets(layers)
+    if dev is None:
+        dev = [DeviceLayer(l, h, sets, torch, bns, nhwc=nhwc) for l, h in zip(layers, inputs)]
+    full = ([DeviceLayer(l, h, sets, torch, bns, full_bn=True, nhwc=nhwc) for l, h in zip(layers, inputs)]
+            if args.full_bn else [])
+
+    def step(i):
+        for d in dev:
+            for _ in range(d.layer.count):
+                d.step(i)
+
+    def full_step(i):
+        for d in full:
+            for _ in range(d.layer.count):
+                d.step(i)
+
+    def runner(fn, nsets=sets):
+        g = capture_steps(torch, fn, nsets) if args.graph else None
+        return (GraphedSteps(g, fn, nsets) if g else fn), g is not None
+
+    step_bytes = sum(l.count * l.algorithmic_bytes() for l in layers)
+    run, graphed = runner(step)
+    for attempt in range(2):
+        ms, clocks, stats = time_steps(torch, dist, run, args.steps, args.warmup, local, world, 30, seconds)
+        if not clocks_rejected(clocks):
+            break
+    res = {"ms_per_step": round(ms, 5), "value": round(whole_job_gbps(step_bytes, world, ms), 1), "timing": stats,
+           "clocks": clocks, "algorithmic_bytes_per_step": step_bytes, "graphed": graphed, "sets": sets}
+    if warm:
+        # the same step on ONE buffer set, back to back: whatever fits in L2 (126 MB) is found there
+        wrun, _ = runner(lambda i: step(0), 1)
+        wms, _, wstats = time_steps(torch, dist, wrun, args.steps, args.warmup, local, world, 30, seconds / 2)
+        res["warm_l2"] = {"ms_per_step": round(wms, 5), "value": round(whole_job_gbps(step_bytes, world, wms), 1),
+                          "min_ms": wstats["min_ms"], "note": "one buffer set reused every step (no rotation)"}
+    layer_info = {}
+    if per_layer:
+        for d in dev:
+            lms, _, lst = time_steps(torch, dist, runner(d.step)[0], args.steps, args.warmup, local, world, 30, layer_seconds)
+            layer_info[d.layer.name] = {"ms": round(lms, 5), "min_ms": lst["min_ms"],
+                                        "gbps": round(d.layer.algorithmic_bytes() / lms / 1e6, 1),
+                                        "algorithmic_bytes": d.layer.algorithmic_bytes(), "count": d.layer.count}
+    if full:
+        fms, _, fst = time_steps(torch, dist, runner(full_step)[0], args.steps, args.warmup, local, world, 30, seconds / 2)
+        fbytes = full_bn_bytes(layers)
+        res["full_bn"] = {"ms_per_step": round(fms, 5), "min_ms": fst["min_ms"], "gbps": round(fbytes / fms / 1e6, 1),
+                          "algorithmic_bytes": fbytes, "speedup_sampled_vs_full": round(fms / ms, 4)}
+        if per_layer:
+            for d in full:
+                lms, _, _ = time_steps(torch, dist, runner(d.step)[0], args.steps, args.warmup, local, world, 30, layer_seconds)
+                layer_info[d.layer.name]["full_bn_ms"] = round(lms, 5)
+                layer_info[d.layer.name]["speedup_vs_full_bn"] = round(lms / layer_info[d.layer.name]["ms"], 4)
+            # the paper's estimation errors (Sec. 5.1, "Correlation Analysis"): E_mu = ||mu_s - mu||_2 and
+            # E_sigma = ||sigma_s - sigma||_2 between the sampled statistics and those of the whole batch,
+            # from the vectors the two forward calls above left behind (diagnostic; synthetic activations)
+            torch.cuda.synchronize()
+            for d, f in zip(dev, full):
+                if d.relu or d.nhwc:
+                    continue                      # that path keeps its statistics in tensors of its own
+                sigma_s, sigma = 1.0 / d.invstd.double(), 1.0 / f.invstd.double()     # sqrt(var + eps) each
+                layer_info[d.layer.name]["estimation_error"] = {
+                    "E_mu": round(float((d.mean.double() - f.mean.double()).norm()), 6),
+                    "E_sigma": round(float((sigma_s - sigma).norm()), 6), "channels": d.layer.C}
+    res["per_layer"] = layer_info
+    return res, dev
+
+
+OTHER_CONFIGS = ["cifar", "vdn", "resnet50", "fs_vdn", "fs_relu"]
 
 
 def run_ours(args):
@@ -422,81 +569,37 @@ def run_ours(args):
         bns.set_tuning(name, int(value))
     layers, seeds = selected_layers(args)
     hosts = [host_inputs(l, s) for l, s in zip(layers, seeds)]
-    bytes_per_tensor_set = sum(4 * l.elems * l.ebytes for l in layers)
-    # rotate buffer sets so that no tensor is reused before > 2x L2 (126 MB) of other data went by
-    sets = 2 if bytes_per_tensor_set >= 512e6 else min(8, max(2, int(np.ceil(512e6 / bytes_per_tensor_set))))
     nhwc = args.layout == "nhwc"
+    peak, peak_source = measured_hbm_peak()
+    sets = buffer_sets(layers)
+
+    # ---- kernel-level events of the library on (K eager steps): the roofline of the dominant kernel
     dev = [DeviceLayer(l, h, sets, torch, bns, nhwc=nhwc) for l, h in zip(layers, hosts)]
-    full = ([DeviceLayer(l, h, sets, torch, bns, full_bn=True, nhwc=nhwc) for l, h in zip(layers, hosts)]
-            if args.full_bn else [])
 
     def step(i):
         for d in dev:
             for _ in range(d.layer.count):
                 d.step(i)
 
-    def full_step(i):
-        for d in full:
-            for _ in range(d.layer.count):
-                d.step(i)
-
-    step_bytes = sum(l.count * l.algorithmic_bytes() for l in layers)
-    # ---- the timed region (kernel-level events of the library on, see roofline below)
-    for attempt in range(2):
-        bns.profile_enable(False)
-        for i in range(args.warmup):     # warm-up outside the profiled window
-            step(i)
-        bns.profile_enable(True)
-        bns.launch_count_reset()
-        ms, clocks = time_steps(torch, dist, step, args.steps, 0, local, world)
-        launches = bns.launch_count()
-        if not clocks_rejected(clocks):
-            break
+    bns.profile_enable(False)
+    for i in range(args.warmup):     # warm-up outside the profiled window
+        step(i)
+    bns.profile_enable(True)
+    bns.launch_count_reset()
+    ms_events, _, _ = time_steps(torch, dist, step, args.steps, 0, local, world)
+    launches = bns.launch_count()
     kernel_times = {}
     for kind in range(bns.KERNEL_KINDS):
         n, tot = bns.profile_read(kind)
         if n:
             kernel_times[bns.kernel_name(kind)] = {"launches": n, "total_ms": round(tot, 4), "avg_us": round(1e3 * tot / n, 3)}
     bns.profile_enable(False)
-    # ---- the same K steps with the library's per-kernel events off: the reported value
-    def runner(fn):
-        g = capture_steps(torch, fn, sets) if args.graph else None
-        return (GraphedSteps(g, fn, sets) if g else fn), g is not None
 
-    run, graphed = runner(step)
-    ms_plain, clocks_plain = time_steps(torch, dist, run, args.steps, args.warmup, local, world)
-    value = whole_job_gbps(step_bytes, world, ms_plain)
-    peak, peak_source = measured_hbm_peak()
-
-    # ---- per-layer numbers and the full-BN comparison (same protocol, each layer alone)
-    per_layer = {}
-    for d in dev:
-        lms, _ = time_steps(torch, dist, runner(d.step)[0], args.steps, args.warmup, local, world)
-        per_layer[d.layer.name] = {"ms": round(lms, 5), "gbps": round(d.layer.algorithmic_bytes() / lms / 1e6, 1),
-                                   "algorithmic_bytes": d.layer.algorithmic_bytes(), "count": d.layer.count}
-    full_info = None
-    if full:
-        fms, _ = time_steps(torch, dist, runner(full_step)[0], args.steps, args.warmup, local, world)
-        # full BN: 3 passes forward + 5 backward; with the fused residual + ReLU 4 + 9 (residual read three times,
-        # dresidual written, the second backward pass re-reads x, residual and dy)
-        fbytes = sum(l.count * ((13 if l.rule == "relu" else 8) * l.elems * l.ebytes + 32 * l.C) for l in layers)
-        full_info = {"ms_per_step": round(fms, 5), "gbps": round(fbytes / fms / 1e6, 1), "algorithmic_bytes": fbytes,
-                     "speedup_sampled_vs_full": round(fms / ms_plain, 4)}
-        for d in full:
-            lms, _ = time_steps(torch, dist, runner(d.step)[0], args.steps, args.warmup, local, world)
-            per_layer[d.layer.name]["full_bn_ms"] = round(lms, 5)
-            per_layer[d.layer.name]["speedup_vs_full_bn"] = round(lms / per_layer[d.layer.name]["ms"], 4)
-        # the paper's estimation errors (Sec. 5.1, "Correlation Analysis"): E_mu = ||mu_s - mu||_2 and
-        # E_sigma = ||sigma_s - sigma||_2 between the sampled statistics and those of the whole batch,
-        # from the vectors the two forward calls above left behind (diagnostic; synthetic activations)
-        torch.cuda.synchronize()
-        for d, f in zip(dev, full):
-            if d.relu or d.nhwc:
-                continue                      # that path keeps its statistics in tensors of its own
-            sigma_s, sigma = 1.0 / d.invstd.double(), 1.0 / f.invstd.double()     # sqrt(var + eps) each
-            per_layer[d.layer.name]["estimation_error"] = {
-                "E_mu": round(float((d.mean.double() - f.mean.double()).norm()), 6),
-                "E_sigma": round(float((sigma_s - sigma).norm()), 6), "channels": d.layer.C}
+    # ---- the reported value: median over >= 30 repetitions of the K steps, per-kernel events off
+    main, dev = measure_workload(torch, dist, bns, args, layers, hosts, local, world, args.seconds, args.seconds / 4,
+                                 dev=dev)
+    ms_plain, value = main["ms_per_step"], main["value"]
+    step_bytes = main["algorithmic_bytes_per_step"]
 
     # ---- roofline of the dominant kernel: backward pass 1 reads dy and x and writes dx (3 E b per launch)
     roofline = None
@@ -507,7 +610,7 @@ def run_ours(args):
         achieved = algo / (kt["avg_us"] * 1e-6) / 1e9
         roofline = {"kernel": "col_bwd_reduce_kernel", "bound": "hbm", "achieved": round(achieved, 1), "peak": peak,
                     "unit": "GB/s", "frac": round(achieved / peak, 4),
-                    "traffic": BWD_REDUCE_DRAM_TRAFFIC_BYTES if args.workload == "resnet18_stage1" else None,
+                    "traffic": BWD_REDUCE_DRAM_TRAFFIC_BYTES if args.workload == "resnet18_stage1" and not args.only else None,
                     "algorithmic_bytes_per_launch": int(algo), "avg_launch_us": kt["avg_us"], "peak_source": peak_source,
                     "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4)}
 
@@ -517,6 +620,25 @@ def run_ours(args):
         e2e = run_e2e(torch, bns, layers, hosts, max(2, min(args.steps, args.e2e_steps)))
     if world > 1:
         dist.barrier()
+
+    # ---- the other configurations of the benchmark spec, each a bounded measurement with its own clock record
+    others = None
+    if args.other_configs and world == 1 and args.workload == "resnet18_stage1" and not args.only and not nhwc:
+        del dev
+        torch.cuda.empty_cache()
+        others = {}
+        for name in OTHER_CONFIGS:
+            olayers = workload_layers(name)
+            oin = [device_inputs(l, layer_seed(name, i), torch) for i, l in enumerate(olayers)]
+            res, odev = measure_workload(torch, dist, bns, args, olayers, oin, local, world, args.seconds / 2,
+                                         args.seconds / 8, warm=name in ("cifar", "vdn"))
+            res["frac_of_hbm_peak"] = round(res["value"] / peak, 4)
+            res["frac_of_nominal_8TBps"] = round(res["value"] / NOMINAL_HBM_GBS, 4)
+            res["layers"] = [f"{l.name}:{l.N}x{l.C}x{l.H}x{l.W}:{l.dtype}:x{l.count}" for l in olayers]
+            res["data"] = "synthetic, drawn on the device with the recipe of the main workload"
+            others[name] = res
+            del odev, oin
+            torch.cuda.empty_cache()
 
     # ---- the oracle on the host cores, bounded sample
     cpu = run_cpu_baseline(layers, hosts, args.cpu_seconds) if (rank == 0 and world == 1 and args.cpu_seconds > 0) else None
@@ -532,14 +654,17 @@ def run_ours(args):
                        "layers": [f"{l.name}:{l.N}x{l.C}x{l.H}x{l.W}:{l.dtype}:x{l.count}" for l in layers],
                        "step": "forward+backward of every layer", "algorithmic_bytes_per_step": step_bytes,
                        "cache": f"inputs larger than L2; {sets} buffer sets rotated", "replicas": world, "layout": args.layout,
-                       "launch": f"CUDA graph replay, {sets} steps per graph" if graphed else "eager launches",
-                       "tuning": args.tune},
+                       "launch": f"CUDA graph replay, {sets} steps per graph" if main["graphed"] else "eager launches",
+                       "value_is": "median over the repetitions of the K-step loop", "tuning": args.tune},
+            "timing": main["timing"], "min_ms_per_step": main["timing"]["min_ms"], "repeats": main["timing"]["repeats"],
+            "warm_l2": main.get("warm_l2"),
             "frac_of_hbm_peak": round(value / world / peak, 4), "hbm_peak_gbs": peak, "hbm_peak_source": peak_source,
             "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
-            "clocks": clocks_plain, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": main["clocks"], "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu,
-            "kernels": kernel_times, "ms_per_step_with_kernel_events": round(ms, 5),
-            "per_layer": per_layer, "full_bn": full_info,
+            "kernels": kernel_times, "ms_per_step_with_kernel_events": round(ms_events, 5),
+            "per_layer": main["per_layer"], "full_bn": main.get("full_bn"),
+            "other_configs": others,
             "paper_context": "overall training speed-up up to 20% (ResNet-18: BS +16.5%, VDN +13.8%, FS +10.7% on 2x V100, "
                              "TensorFlow); not comparable to a kernel GB/s",
         }
@@ -687,7 +812,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="resnet18_stage1",
@@ -701,6 +826,10 @@ def main():
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="time eager launches instead of replaying a CUDA graph of the step")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--seconds", type=float, default=0.6,
+                    help="least duration of the main timed region (the K-step loop is repeated, 30 times at least)")
+    ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
+                    help="skip the bounded measurements of the other configurations (CIFAR sweep, VDN, ResNet-50 sweep, ...)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the oracle baseline (0 = skip)")
     args = ap.parse_args()

@@ -649,15 +649,17 @@ col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::stor
     typename T::storage* yp = y + p;
     // x is an input of the whole call, so the first rows can be requested before the statistics
     // kernels ahead of this one have finished; only mean / invstd have to wait for them.
+    // Rows go in batches of kUnroll with all loads of a batch in flight together; the last batch may be short.
     int i = ck;
-    const bool head = p < P && i + (kUnroll - 1) * nchunks < order.rows;
     Vec<T, V> v[kUnroll];
     int row[kUnroll];
-    if (head) {
+    if (p < P) {
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-            row[u] = order(i + u * nchunks);
-            v[u].load(xp + static_cast<size_t>(row[u]) * P);
+            if (i + u * nchunks < order.rows) {
+                row[u] = order(i + u * nchunks);
+                v[u].load(xp + static_cast<size_t>(row[u]) * P);
+            }
         }
     }
     grid_dependency_wait();
@@ -673,35 +675,24 @@ col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::stor
             b[j] = fmaf(-mean[c[j]], a[j], beta[c[j]]);
         }
     }
-    if (head) {
+    while (true) {
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
+            if (i + u * nchunks < order.rows) {
 #pragma unroll
-            for (int j = 0; j < V; ++j) v[u].set(j, fmaf(a[j], v[u].get(j), b[j]));
-            v[u].store(yp + static_cast<size_t>(row[u]) * P);
+                for (int j = 0; j < V; ++j) v[u].set(j, fmaf(a[j], v[u].get(j), b[j]));
+                v[u].store(yp + static_cast<size_t>(row[u]) * P);
+            }
         }
         i += kUnroll * nchunks;
-    }
-    for (; i + (kUnroll - 1) * nchunks < order.rows; i += kUnroll * nchunks) {
+        if (i >= order.rows) break;
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-            row[u] = order(i + u * nchunks);
-            v[u].load(xp + static_cast<size_t>(row[u]) * P);
+            if (i + u * nchunks < order.rows) {
+                row[u] = order(i + u * nchunks);
+                v[u].load(xp + static_cast<size_t>(row[u]) * P);
+            }
         }
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-#pragma unroll
-            for (int j = 0; j < V; ++j) v[u].set(j, fmaf(a[j], v[u].get(j), b[j]));
-            v[u].store(yp + static_cast<size_t>(row[u]) * P);
-        }
-    }
-    for (; i < order.rows; i += nchunks) {
-        const size_t off = static_cast<size_t>(order(i)) * P;
-        Vec<T, V> w;
-        w.load(xp + off);
-#pragma unroll
-        for (int j = 0; j < V; ++j) w.set(j, fmaf(a[j], w.get(j), b[j]));
-        w.store(yp + off);
     }
 }
 
