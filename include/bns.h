@@ -75,7 +75,9 @@ typedef struct {
     int offset_mode;            /* bns_offset_mode                                                */
     const int32_t* offsets;     /* (oh,ow) int32 pairs, oh in [0,H-ph], ow in [0,W-pw]:           */
                                 /* SHARED: HOST, 1 pair (validated on the host);                  */
-                                /* PER_SAMPLE: DEVICE, N pairs; PER_MAP: DEVICE, N*C pairs.       */
+                                /* PER_SAMPLE: DEVICE, N pairs; PER_MAP: DEVICE, N*C pairs - the  */
+                                /* caller guarantees that many: the kernels index the array by    */
+                                /* sample (and channel) and cannot check its length.              */
                                 /* Device-resident pairs are checked by the kernels: a pair out   */
                                 /* of range is clamped into range and BNS_FLAG_BAD_OFFSET is set  */
                                 /* in the workspace status word (see bns_workspace_status)        */
@@ -263,7 +265,9 @@ bns_status bns_backward_nhwc(const bns_shape* shape, const void* x, const void* 
  *  - A shape/rule whose bns_workspace_bytes() exceeds bns_static_workspace_bytes() is rejected with
  *    BNS_ERR_WORKSPACE before anything is launched (the ResNet-50 layers at N=256 need up to 2.6 MB).
  *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
- *    that device current) and keeps it; make that first call before any stream capture begins.
+ *    that device current) and keeps it for the life of the process (the device's primary context is
+ *    assumed to live that long; after a cudaDeviceReset the kept address is stale).  Host threads may
+ *    make that first call at the same time.  Make it before any stream capture begins.
  *  - All calls on a device share the one array, which keeps whatever the previous call left in it.
  *    Nothing in it needs to start at zero (the status word is cleared by the call when it is used),
  *    but two calls that overlap in time on the same GPU - different streams, or different host

@@ -1715,12 +1715,15 @@ static __device__ __align__(256) unsigned char g_static_workspace[BNS_STATIC_WOR
 
 namespace {
 void* g_static_workspace_address[kMaxDevices] = {};  // resolved by the first call made on each device
+std::mutex g_static_workspace_mutex;                 // host threads may make that first call together
 
-// Device address of the static scratch on the device that is current now.
+// Device address of the static scratch on the device that is current now.  The address is kept for the
+// life of the process: it belongs to the device's primary context, which is assumed to live that long.
 bns_status static_workspace_address(void** address) {
     int device = -1;
     if (cudaGetDevice(&device) != cudaSuccess) return BNS_ERR_CUDA;
     if (device < 0 || device >= kMaxDevices) return BNS_ERR_CUDA;
+    std::lock_guard<std::mutex> guard(g_static_workspace_mutex);
     if (!g_static_workspace_address[device]) {
         void* p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return BNS_ERR_CUDA;

@@ -35,7 +35,11 @@ def test_status_strings():
 
 def _call_forward(shape, sp, x=0x1000, gamma=0x2000, beta=0x3000, y=0x4000, mean=0x5000, invstd=0x6000, eps=1e-5,
                   ws=0x10000, ws_bytes=1 << 30):
-    """Fake, never dereferenced device addresses: every case below must be refused on the host."""
+    """Fake, never dereferenced device addresses: every case below must be refused on the host.  Run only
+    where no GPU is visible, so that a check that stopped working cannot send a kernel to a wild address."""
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("fake device addresses are only used where no GPU can be reached")
     lib = bns.load()
     sh = bns._Shape(*shape)
     return lib.bns_forward(ctypes.byref(sh), x, gamma, beta, eps, ctypes.byref(sp), y, mean, invstd, ws, ws_bytes, None)
@@ -91,3 +95,23 @@ def test_binding_refuses_cpu_tensors():
     with pytest.raises(TypeError):
         bns.forward(x, torch.ones(3), torch.zeros(3), 1e-5, bns.Sampling.full(),
                     workspace=torch.empty(1 << 20, dtype=torch.uint8))
+
+
+def test_binding_checks_the_length_of_device_offsets():
+    """Per-sample / per-map patch offsets are indexed by sample (and channel) on the device, so the binding
+    refuses a tensor that does not hold one pair for each.  (Checked before anything touches the tensor's
+    memory, so an object standing in for a CUDA tensor serves on a machine without a GPU.)"""
+    import torch
+
+    class FakeCudaInt32(torch.Tensor):
+        is_cuda = True
+
+    def offsets(pairs):
+        return torch.zeros(pairs, 2, dtype=torch.int32).as_subclass(FakeCudaInt32)
+
+    shape = bns._Shape(8, 16, 8, 8, bns.F32)
+    bns.Sampling.feature(2, 2, offsets(8), bns.OFF_PER_SAMPLE)._c(shape)
+    bns.Sampling.feature(2, 2, offsets(8 * 16), bns.OFF_PER_MAP)._c(shape)
+    for mode, pairs in ((bns.OFF_PER_SAMPLE, 7), (bns.OFF_PER_SAMPLE, 8 * 16), (bns.OFF_PER_MAP, 8), (bns.OFF_PER_MAP, 127)):
+        with pytest.raises(TypeError):
+            bns.Sampling.feature(2, 2, offsets(pairs), mode)._c(shape)

@@ -17,6 +17,15 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("dtype,dims", [("f32", (40, 24, 20, 20)), ("bf16", (32, 48, 14, 14)), ("f32", (9, 5, 7, 7))])
 @pytest.mark.parametrize("mix,with_dyv", [(0.5, True), (0.25, False)])
 def test_mixed_statistics_forward_backward(rule, kw, dtype, dims, mix, with_dyv):
+    _check_mixed(rule, kw, dtype, dims, mix, with_dyv)
+
+
+def test_mixed_statistics_at_benchmark_size():
+    """The shape and rule that bench.py times as `fs_vdn`: 256x64x56x56 fp32, 8x8 patch, two virtual samples."""
+    _check_mixed("feature", dict(ph=8, pw=8, offset_mode=0), "f32", (256, 64, 56, 56), 0.5, False)
+
+
+def _check_mixed(rule, kw, dtype, dims, mix, with_dyv):
     import torch
     from paper_1810_10962_b200 import bns
     case = make_case(*dims, rule, seed=93, dtype=dtype, **kw)
@@ -185,6 +194,37 @@ def test_fused_residual_relu(rule, kw, dtype, dims, with_residual):
         assert dres is None
 
 
+def test_fused_residual_relu_at_benchmark_size():
+    """The shape and rule that bench.py times as `fs_relu`: 256x64x56x56 fp32, 8x8 patch, with a residual.  At
+    51 million elements some pre-activation always lands within rounding of zero, where the rectifier's mask
+    is either side's to decide; so the residual is nudged, using the oracle's own pre-activations only, until
+    every one of them is well away from zero.  Then the masks agree and every element is compared."""
+    import torch
+    from paper_1810_10962_b200 import bns
+    case = make_case(256, 64, 56, 56, "feature", seed=98, ph=8, pw=8, offset_mode=0)
+    osp = case.oracle_sampling()
+    res_np = I.upstream_gradient(case.x.shape, 98, I.TAG_XV)
+    f = O.forward_relu(case.x, res_np, case.gamma, case.beta, case.eps, osp)
+    near = np.abs(f.z) < 1e-3
+    res_np = np.where(near, res_np + np.float32(0.0625), res_np).astype(np.float32)
+    f = O.forward_relu(case.x, res_np, case.gamma, case.beta, case.eps, osp)
+    assert np.abs(f.z).min() > 5e-4
+    b, dres_want = O.backward_relu(case.x, case.dy, case.gamma, f, case.eps, osp)
+    x, dy, res = _to_device(case.x, "f32"), _to_device(case.dy, "f32"), _to_device(res_np, "f32")
+    gamma, beta = torch.from_numpy(case.gamma).cuda(), torch.from_numpy(case.beta).cuda()
+    sp = gpu_sampling(case)
+    y, mean, invstd = bns.forward_relu(x, res, gamma, beta, case.eps, sp)
+    dx, dres, dgamma, dbeta = bns.backward_relu(x, res, dy, gamma, beta, mean, invstd, sp)
+    torch.cuda.synchronize()
+    close_f32(mean.cpu().numpy(), f.mean, "mean")
+    close_f32(invstd.cpu().numpy(), f.invstd, "invstd")
+    close_f32(_to_host(y), f.y, "y")
+    close_f32(_to_host(dx), b.dx, "dx")
+    close_f32(dgamma.cpu().numpy(), b.dgamma, "dgamma")
+    close_f32(dbeta.cpu().numpy(), b.dbeta, "dbeta")
+    assert np.array_equal(_to_host(dres), dres_want.astype(np.float32))
+
+
 def _nhwc(a):
     return np.ascontiguousarray(np.transpose(a, (0, 2, 3, 1)))
 
@@ -205,6 +245,19 @@ NHWC_CASES = [
                                         ("bf16", (3, 2080, 2, 2)), ("f32", (40, 16, 16, 16))])
 def test_channels_last_layout(rule, kw, dtype, dims):
     """The NHWC entry points against the (NCHW) oracle on the transposed tensors."""
+    _check_channels_last(rule, kw, dtype, dims)
+
+
+@pytest.mark.parametrize("rule,kw,dtype,dims", [
+    ("batch", dict(k=32), "f32", (256, 64, 56, 56)),                            # bench.py --layout nhwc, first layer
+    ("feature", dict(ph=8, pw=8, offset_mode=0), "f32", (256, 64, 56, 56)),     # ... and second: 802 816 rows
+    ("feature", dict(ph=1, pw=1, offset_mode=0), "bf16", (256, 256, 14, 14)),   # a ResNet-50 layer
+])
+def test_channels_last_layout_at_benchmark_size(rule, kw, dtype, dims):
+    _check_channels_last(rule, kw, dtype, dims)
+
+
+def _check_channels_last(rule, kw, dtype, dims):
     import torch
     from paper_1810_10962_b200 import bns
     kw = dict(kw)
