@@ -186,29 +186,35 @@ bns_status bns_inference_forward(const bns_shape* shape, const void* x, const fl
  *   bns_sync_local_moments   this rank's sampled set -> moments[3][C] = (count, mean, M2) rows
  *   (all-gather the 3C floats of every rank into [ranks][3][C])
  *   bns_sync_merge_moments   merges the ranks' rows in rank order (same bits on every rank) -> mean, invstd
+ *                            and, if count is not NULL, count[C] = sampled points per channel over all ranks
  *   bns_sync_normalize       Eq. 1 on this rank's x with the shared statistics
  *   bns_sync_backward_sums   sums[2][C] = (sum dy, sum dy xhat) over this rank's elements, and
  *                            dx = gamma invstd dy for every element (lower branch of Eq. 6);
  *                            the two rows are also this rank's share of dbeta and dgamma
  *   (all-reduce the 2C floats)
  *   bns_sync_backward_apply  upper branch of Eq. 6 on this rank's sampled elements with the summed
- *                            rows and sampled_total = the number of sampled points per channel over
- *                            all ranks
- * rule may be FULL, BATCH or FEATURE (VIRTUAL: feed the virtual samples to one rank as a BATCH rule
- * over them).  Workspace as for bns_forward with the same shape and rule (FULL for _backward_sums).
+ *                            rows and the merged count (DEVICE float[C]: the count never visits the host)
+ *
+ * The three variants of the paper's list are all expressible: (1) every rank samples its slice by the
+ * same rule (FULL, BATCH or FEATURE); (2) only a fraction of the ranks contributes statistics - the
+ * others pass sampling = NULL to _local_moments (a count of zero, which the merge passes over) and to
+ * _backward_apply (nothing to correct); (3) the virtual samples are fed to one rank - that rank passes
+ * a VIRTUAL rule (xv, optionally dyv / dxv) to _local_moments, to _backward_sums as `virtual_rows` (their
+ * gradient joins its sums when dyv is given) and to _backward_apply (which writes dxv), the others NULL.
+ * Workspace as for bns_forward with the same shape and rule (FULL where sampling is NULL).
  */
 bns_status bns_sync_local_moments(const bns_shape* shape, const void* x, const bns_sampling* sampling, float eps,
                                   float* moments, void* workspace, size_t workspace_bytes, void* cuda_stream);
 bns_status bns_sync_merge_moments(int C, int ranks, const float* moments, float eps, float* mean, float* invstd,
-                                  void* cuda_stream);
+                                  float* count, void* cuda_stream);
 bns_status bns_sync_normalize(const bns_shape* shape, const void* x, const float* gamma, const float* beta,
                               const float* mean, const float* invstd, void* y, void* cuda_stream);
 bns_status bns_sync_backward_sums(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
-                                  const float* mean, const float* invstd, void* dx, float* sums,
-                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+                                  const float* mean, const float* invstd, const bns_sampling* virtual_rows,
+                                  void* dx, float* sums, void* workspace, size_t workspace_bytes, void* cuda_stream);
 bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
                                    const float* mean, const float* invstd, const bns_sampling* sampling,
-                                   const float* sums, double sampled_total, void* dx,
+                                   const float* sums, const float* count, void* dx,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*

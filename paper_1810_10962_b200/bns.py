@@ -126,13 +126,13 @@ def load():
     lib.bns_sync_local_moments.restype = ctypes.c_int
     lib.bns_sync_local_moments.argtypes = [shp, vp, smp, fl, vp, vp, sz, vp]
     lib.bns_sync_merge_moments.restype = ctypes.c_int
-    lib.bns_sync_merge_moments.argtypes = [ctypes.c_int, ctypes.c_int, vp, fl, vp, vp, vp]
+    lib.bns_sync_merge_moments.argtypes = [ctypes.c_int, ctypes.c_int, vp, fl, vp, vp, vp, vp]
     lib.bns_sync_normalize.restype = ctypes.c_int
     lib.bns_sync_normalize.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp]
     lib.bns_sync_backward_sums.restype = ctypes.c_int
-    lib.bns_sync_backward_sums.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.bns_sync_backward_sums.argtypes = [shp, vp, vp, vp, vp, vp, smp, vp, vp, vp, sz, vp]
     lib.bns_sync_backward_apply.restype = ctypes.c_int
-    lib.bns_sync_backward_apply.argtypes = [shp, vp, vp, vp, vp, vp, smp, vp, ctypes.c_double, vp, vp, sz, vp]
+    lib.bns_sync_backward_apply.argtypes = [shp, vp, vp, vp, vp, vp, smp, vp, vp, vp, vp, sz, vp]
     lib.bns_forward_relu.restype = ctypes.c_int
     lib.bns_forward_relu.argtypes = [shp, vp, vp, vp, vp, fl, smp, vp, vp, vp, vp, sz, vp]
     lib.bns_backward_relu.restype = ctypes.c_int
@@ -504,11 +504,17 @@ def inference_forward(x, gamma, beta, eps, mean_ma, var_ma, y=None, workspace=No
 
 
 # ----------------------------------------------------------------------------- statistics shared by several GPUs
-def sync_local_moments(x, sampling: Sampling, eps, workspace=None):
-    """bns_sync_local_moments: float32 [3, C] = (count, mean, M2) of this rank's sampled set."""
+def sync_local_moments(x, sampling: Optional[Sampling], eps, workspace=None):
+    """bns_sync_local_moments: float32 [3, C] = (count, mean, M2) of this rank's sampled set; ``sampling=None``
+    means that this rank contributes nothing (a count of zero)."""
     sh = _shape(x)
-    sp = sampling._c(sh)
     moments = torch.empty(3, x.shape[1], dtype=torch.float32, device=x.device)
+    if sampling is None:
+        _check(load().bns_sync_local_moments(ctypes.byref(sh), _dev(x), None, float(eps), moments.data_ptr(), None, 0,
+                                             _stream()), "bns_sync_local_moments")
+        return moments
+    _check_virtual(x, sampling)
+    sp = sampling._c(sh)
     ws, wp, wn = _workspace(x, sampling, workspace)
     _check(load().bns_sync_local_moments(ctypes.byref(sh), _dev(x), ctypes.byref(sp), float(eps), moments.data_ptr(),
                                          wp, wn, _stream()), "bns_sync_local_moments")
@@ -516,13 +522,14 @@ def sync_local_moments(x, sampling: Sampling, eps, workspace=None):
 
 
 def sync_merge_moments(gathered, eps):
-    """bns_sync_merge_moments on a [ranks, 3, C] tensor (an all-gather result): returns (mean, invstd)."""
+    """bns_sync_merge_moments on a [ranks, 3, C] tensor (an all-gather result): returns (mean, invstd, count),
+    count being the sampled points per channel over all ranks (it stays on the device)."""
     R, three, C = gathered.shape
     assert three == 3 and gathered.dtype == torch.float32
-    mean, invstd = (torch.empty(C, dtype=torch.float32, device=gathered.device) for _ in range(2))
+    mean, invstd, count = (torch.empty(C, dtype=torch.float32, device=gathered.device) for _ in range(3))
     _check(load().bns_sync_merge_moments(C, R, _dev(gathered), float(eps), mean.data_ptr(), invstd.data_ptr(),
-                                         _stream()), "bns_sync_merge_moments")
-    return mean, invstd
+                                         count.data_ptr(), _stream()), "bns_sync_merge_moments")
+    return mean, invstd, count
 
 
 def sync_normalize(x, gamma, beta, mean, invstd, y=None):
@@ -534,27 +541,39 @@ def sync_normalize(x, gamma, beta, mean, invstd, y=None):
     return y
 
 
-def sync_backward_sums(x, dy, gamma, mean, invstd, dx=None, workspace=None):
-    """bns_sync_backward_sums: returns (dx without the statistics terms, sums float32 [2, C])."""
+def sync_backward_sums(x, dy, gamma, mean, invstd, dx=None, workspace=None, virtual_rows: Optional[Sampling] = None):
+    """bns_sync_backward_sums: returns (dx without the statistics terms, sums float32 [2, C]).  ``virtual_rows``
+    is the VIRTUAL rule of the rank that fed virtual samples into the statistics: with dyv set, their gradient
+    joins this rank's sums."""
     sh = _shape(x)
     C = x.shape[1]
     dx = torch.empty_like(x) if dx is None else dx
     sums = torch.empty(2, C, dtype=torch.float32, device=x.device)
-    ws, wp, wn = _workspace(x, Sampling.full(), workspace)
+    rule = virtual_rows if (virtual_rows is not None and virtual_rows.dyv is not None) else Sampling.full()
+    ws, wp, wn = _workspace(x, rule, workspace)
+    vp = None
+    if virtual_rows is not None:
+        _check_virtual(x, virtual_rows)
+        vr = virtual_rows._c(sh)
+        vp = ctypes.byref(vr)
     _check(load().bns_sync_backward_sums(ctypes.byref(sh), _dev(x), _dev(dy), _vec(gamma, C), _vec(mean, C),
-                                         _vec(invstd, C), _dev(dx), sums.data_ptr(), wp, wn, _stream()),
+                                         _vec(invstd, C), vp, _dev(dx), sums.data_ptr(), wp, wn, _stream()),
            "bns_sync_backward_sums")
     return dx, sums
 
 
-def sync_backward_apply(x, dy, gamma, mean, invstd, sampling: Sampling, sums, sampled_total, dx, workspace=None):
-    """bns_sync_backward_apply: adds the statistics terms to dx on this rank's sampled elements."""
+def sync_backward_apply(x, dy, gamma, mean, invstd, sampling: Optional[Sampling], sums, count, dx, workspace=None):
+    """bns_sync_backward_apply: adds the statistics terms to dx on this rank's sampled elements (for a VIRTUAL
+    rule: writes dxv).  ``count`` is the merged count from sync_merge_moments; ``sampling=None``: nothing to do."""
     sh = _shape(x)
-    sp = sampling._c(sh)
     C = x.shape[1]
+    if sampling is None:
+        return dx
+    _check_virtual(x, sampling)
+    sp = sampling._c(sh)
     ws, wp, wn = _workspace(x, sampling, workspace)
     _check(load().bns_sync_backward_apply(ctypes.byref(sh), _dev(x), _dev(dy), _vec(gamma, C), _vec(mean, C),
-                                          _vec(invstd, C), ctypes.byref(sp), _dev(sums), float(sampled_total), _dev(dx),
+                                          _vec(invstd, C), ctypes.byref(sp), _dev(sums), _vec(count, C), _dev(dx),
                                           wp, wn, _stream()), "bns_sync_backward_apply")
     return dx
 

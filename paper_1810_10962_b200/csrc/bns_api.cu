@@ -1492,10 +1492,19 @@ bns_status bns_inference_forward(const bns_shape* shape, const void* x, const fl
 // ---------------------------------------------------------------------------------------- statistics shared by several GPUs
 bns_status bns_sync_local_moments(const bns_shape* shape, const void* x, const bns_sampling* sampling, float eps,
                                   float* moments, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!sampling) {
+        // this rank samples nothing: a count of zero, which the merge passes over
+        bns_status sc = check_shape(shape);
+        if (sc != BNS_OK) return sc;
+        if (!moments) return BNS_ERR_NULL;
+        return cudaMemsetAsync(moments, 0, 3 * static_cast<size_t>(shape->C) * sizeof(float),
+                               static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+                   ? BNS_OK
+                   : BNS_ERR_CUDA;
+    }
     Problem pb;
     bns_status st = make_problem(shape, sampling, pb);
     if (st != BNS_OK) return st;
-    if (pb.rule == BNS_RULE_VIRTUAL) return BNS_ERR_RULE;
     if (!x || !moments) return BNS_ERR_NULL;
     if (!(eps > 0.f)) return BNS_ERR_SHAPE;
     if (!aligned16(x)) return BNS_ERR_ALIGN;
@@ -1510,11 +1519,11 @@ bns_status bns_sync_local_moments(const bns_shape* shape, const void* x, const b
 }
 
 bns_status bns_sync_merge_moments(int C, int ranks, const float* moments, float eps, float* mean, float* invstd,
-                                  void* cuda_stream) {
+                                  float* count, void* cuda_stream) {
     if (C <= 0 || ranks <= 0 || !(eps > 0.f)) return BNS_ERR_SHAPE;
     if (!moments || !mean || !invstd) return BNS_ERR_NULL;
     launch(BNS_KERNEL_VECTOR, merge_rank_moments_kernel, per_channel_grid(C), static_cast<cudaStream_t>(cuda_stream),
-           moments, ranks, C, eps, mean, invstd);
+           moments, ranks, C, eps, mean, invstd, count);
     return last_error();
 }
 
@@ -1536,11 +1545,13 @@ bns_status bns_sync_normalize(const bns_shape* shape, const void* x, const float
 }
 
 bns_status bns_sync_backward_sums(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
-                                  const float* mean, const float* invstd, void* dx, float* sums, void* workspace,
-                                  size_t workspace_bytes, void* cuda_stream) {
-    bns_sampling sp = full_rule();
+                                  const float* mean, const float* invstd, const bns_sampling* virtual_rows, void* dx,
+                                  float* sums, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    bns_sampling full = full_rule();
+    if (virtual_rows && virtual_rows->rule != BNS_RULE_VIRTUAL) return BNS_ERR_RULE;
+    const bool with_virtual = virtual_rows && virtual_rows->dyv;
     Problem pb;
-    bns_status st = make_problem(shape, &sp, pb);
+    bns_status st = make_problem(shape, with_virtual ? virtual_rows : &full, pb);
     if (st != BNS_OK) return st;
     if (!x || !dy || !gamma || !mean || !invstd || !dx || !sums) return BNS_ERR_NULL;
     if (!aligned16(x) || !aligned16(dy) || !aligned16(dx)) return BNS_ERR_ALIGN;
@@ -1548,33 +1559,44 @@ bns_status bns_sync_backward_sums(const bns_shape* shape, const void* x, const v
     if (st != BNS_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const ColPlan& pl = pb.main_plan;
-    // row 0: sum dy (dbeta), row 1: sum dy xhat (dgamma) over this rank's elements
-    GradSink sink{ws_at<float2>(workspace, pb.off_bwd), pl.layout(), nullptr, pl.layout(), invstd, sums + pb.C, sums};
+    const ColPlan& pv = pb.stat_plan;
+    // row 0: sum dy (dbeta), row 1: sum dy xhat (dgamma) over this rank's elements (and its virtual rows)
+    GradSink sink{ws_at<float2>(workspace, pb.off_bwd), pl.layout(),
+                  with_virtual ? ws_at<float2>(workspace, pb.off_bwd_v) : nullptr, pv.layout(), invstd, sums + pb.C, sums};
     BNS_BY_TYPE_V(pb.dtype, pl.V,
                   (launch(BNS_KERNEL_BWD_REDUCE, bwd_reduce_variant<T, V, true>(pb.HW), pl.grid(), stream, in<T>(x), in<T>(dy),
                           out<T>(dx), gamma, mean, invstd, RowOrder{RowOrder::kIdentity, pb.N, 0, 0}, pl.nchunks, pl.tiles,
                           pb.HW, pb.P, false, sink)));
+    if (with_virtual)
+        BNS_BY_TYPE_V(virtual_rows->xv_dtype, pv.V,
+                      (launch(BNS_KERNEL_BWD_REDUCE, bwd_reduce_variant<T, V, false>(pb.HW), pv.grid(), stream,
+                              in<T>(virtual_rows->xv), in<T>(virtual_rows->dyv), out<T>(nullptr), gamma, mean, invstd,
+                              RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P, true, sink)));
     launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
     return last_error();
 }
 
 bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
                                    const float* mean, const float* invstd, const bns_sampling* sampling,
-                                   const float* sums, double sampled_total, void* dx, void* workspace,
+                                   const float* sums, const float* count, void* dx, void* workspace,
                                    size_t workspace_bytes, void* cuda_stream) {
+    if (!sampling) return check_shape(shape);  // nothing of this rank is in the sampled set: dx stays as it is
     Problem pb;
     bns_status st = make_problem(shape, sampling, pb);
     if (st != BNS_OK) return st;
-    if (pb.rule == BNS_RULE_VIRTUAL) return BNS_ERR_RULE;
-    if (!x || !dy || !gamma || !mean || !invstd || !sums || !dx) return BNS_ERR_NULL;
-    if (!(sampled_total >= pb.s)) return BNS_ERR_SHAPE;  // the shared set holds at least this rank's share
+    if (!x || !dy || !gamma || !mean || !invstd || !sums || !count || !dx) return BNS_ERR_NULL;
     if (!aligned16(x) || !aligned16(dy) || !aligned16(dx)) return BNS_ERR_ALIGN;
     st = check_workspace(pb, workspace, workspace_bytes);
     if (st != BNS_OK) return st;
+    if (pb.total - pb.off_stats < 2 * static_cast<size_t>(pb.C) * sizeof(float)) return BNS_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const float* dbeta = sums;
-    const float* dgamma = sums + pb.C;
-    const float inv_s = static_cast<float>(1.0 / sampled_total);
+    // the summed rows divided by the sampled count of all ranks, which stays on the device: the fix-up
+    // kernels then run with 1/s = 1
+    float* shares = ws_at<float>(workspace, pb.off_stats);
+    launch(BNS_KERNEL_VECTOR, per_point_shares_kernel, per_channel_grid(pb.C), stream, sums, count, pb.C, shares);
+    const float* dbeta = shares;
+    const float* dgamma = shares + pb.C;
+    const float inv_s = 1.0f;
     const ColPlan& pl = pb.main_plan;
     const ColPlan& pv = pb.stat_plan;
     if (pb.rule == BNS_RULE_FULL) {
@@ -1590,7 +1612,7 @@ bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const 
                       (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(x), in<T>(dy),
                               out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, list, pb.begin,
                               RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P)));
-    } else {
+    } else if (pb.rule == BNS_RULE_FEATURE) {
         unsigned* status;
         st = clear_status(pb, workspace, stream, &status);
         if (st != BNS_OK) return st;
@@ -1598,6 +1620,13 @@ bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const 
         BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, patch_fixup_kernel<T>, pp.grid(), stream, in<T>(x), in<T>(dy),
                                       out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, pb.patch, pb.N, pb.C, pb.H,
                                       pb.W, pp.nchunks, pp.tiles, status)));
+    } else if (sampling->dxv) {
+        // the virtual samples that this rank fed into the statistics: every one of them takes the upper branch
+        BNS_BY_TYPE_V(sampling->xv_dtype, pv.V,
+                      (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(sampling->xv),
+                              in<T>(sampling->dyv), out<T>(sampling->dxv), gamma, mean, invstd, dgamma, dbeta, inv_s,
+                              static_cast<const int*>(nullptr), 0, RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks,
+                              pv.tiles, pb.HW, pb.P)));
     }
     return last_error();
 }

@@ -1187,7 +1187,7 @@ moments_rows_kernel(float* __restrict__ rows, float count, float eps, int C) {
 // Merges the (count, mean, M2) rows of R ranks (rank-major: [R][3][C]) in rank order.
 __global__ void __launch_bounds__(kThreads)
 merge_rank_moments_kernel(const float* __restrict__ rows, int R, int C, float eps, float* __restrict__ mean,
-                          float* __restrict__ invstd) {
+                          float* __restrict__ invstd, float* __restrict__ count) {
     grid_dependency_wait();
     grid_dependency_launch();
     const int c = blockIdx.x * kThreads + threadIdx.x;
@@ -1199,6 +1199,20 @@ merge_rank_moments_kernel(const float* __restrict__ rows, int R, int C, float ep
     }
     mean[c] = acc.mean;
     invstd[c] = 1.0f / sqrtf(acc.m2 / acc.cnt + eps);
+    if (count) count[c] = acc.cnt;  // sampled points per channel over all ranks
+}
+
+// The summed backward rows (sum dy, sum dy xhat) of all ranks divided by the merged sampled count: the
+// per-point shares that the upper branch of Eq. 6 subtracts.
+__global__ void __launch_bounds__(kThreads)
+per_point_shares_kernel(const float* __restrict__ sums, const float* __restrict__ count, int C, float* __restrict__ shares) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x * kThreads + threadIdx.x;
+    if (c >= C) return;
+    const float inv = 1.0f / count[c];
+    shares[c] = sums[c] * inv;
+    shares[C + c] = sums[C + c] * inv;
 }
 
 // ------------------------------------------------------------------------------------ BN + residual add + ReLU

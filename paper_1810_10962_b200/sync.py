@@ -29,20 +29,26 @@ def all_reduce_rows(rows: torch.Tensor, group=None) -> torch.Tensor:
     return total
 
 
-def forward(x, gamma, beta, eps, sampling: bns.Sampling, group=None):
-    """Returns (y, mean, invstd, sampled_total): statistics of the union of all ranks' sampled sets."""
+def forward(x, gamma, beta, eps, sampling, group=None):
+    """Returns (y, mean, invstd, count): statistics of the union of all ranks' sampled sets and the number of
+    sampled points per channel in that union (a device tensor; nothing is read back to the host).
+    ``sampling`` is this rank's rule - FULL, BATCH or FEATURE on its slice, a VIRTUAL rule on the one rank that
+    is fed the virtual samples, or None on a rank that contributes no statistics."""
     local = bns.sync_local_moments(x, sampling, eps)
     gathered = all_gather_rows(local, group)
-    mean, invstd = bns.sync_merge_moments(gathered, eps)
+    mean, invstd, count = bns.sync_merge_moments(gathered, eps)
     y = bns.sync_normalize(x, gamma, beta, mean, invstd)
-    sampled_total = float(gathered[:, 0, 0].sum().item())
-    return y, mean, invstd, sampled_total
+    if sampling is not None and sampling.rule == bns.RULE_VIRTUAL and sampling.yv is not None:
+        bns.sync_normalize(sampling.xv, gamma, beta, mean, invstd, y=sampling.yv)
+    return y, mean, invstd, count
 
 
-def backward(x, dy, gamma, mean, invstd, sampling: bns.Sampling, sampled_total, group=None):
+def backward(x, dy, gamma, mean, invstd, sampling, count, group=None):
     """Returns (dx, dgamma_local, dbeta_local): dx uses the sums of all ranks; the parameter gradients are
-    this rank's share (a data-parallel wrapper reduces them with the other gradients)."""
-    dx, local = bns.sync_backward_sums(x, dy, gamma, mean, invstd)
+    this rank's share (a data-parallel wrapper reduces them with the other gradients).  On the rank that holds
+    virtual samples their gradient dyv joins the sums and dxv is written."""
+    virtual = sampling if (sampling is not None and sampling.rule == bns.RULE_VIRTUAL) else None
+    dx, local = bns.sync_backward_sums(x, dy, gamma, mean, invstd, virtual_rows=virtual)
     total = all_reduce_rows(local, group)
-    bns.sync_backward_apply(x, dy, gamma, mean, invstd, sampling, total, sampled_total, dx)
+    bns.sync_backward_apply(x, dy, gamma, mean, invstd, sampling, total, count, dx)
     return dx, local[1], local[0]

@@ -130,15 +130,55 @@ def test_statistics_shared_by_several_ranks_equal_one_big_batch(rule, dtype, ran
     else:
         osp = O.Sampling.full()
         sps = [bns.Sampling.full() for _ in range(ranks)]
-    s_total = O.sample_count(N, H, W, osp)
     xs = [_to_device(x_np[r * n_local:(r + 1) * n_local], dtype) for r in range(ranks)]
     dys = [_to_device(dy_np[r * n_local:(r + 1) * n_local], dtype) for r in range(ranks)]
     gathered = torch.stack([bns.sync_local_moments(xs[r], sps[r], eps) for r in range(ranks)])   # "all-gather"
-    mean, invstd = bns.sync_merge_moments(gathered, eps)
+    mean, invstd, count = bns.sync_merge_moments(gathered, eps)
     ys = [bns.sync_normalize(xs[r], gamma, beta, mean, invstd) for r in range(ranks)]
     partial = [bns.sync_backward_sums(xs[r], dys[r], gamma, mean, invstd) for r in range(ranks)]
     sums = torch.stack([p[1] for p in partial]).sum(dim=0)                                        # "all-reduce"
-    dxs = [bns.sync_backward_apply(xs[r], dys[r], gamma, mean, invstd, sps[r], sums, s_total, partial[r][0])
+    dxs = [bns.sync_backward_apply(xs[r], dys[r], gamma, mean, invstd, sps[r], sums, count, partial[r][0])
+           for r in range(ranks)]
+    torch.cuda.synchronize()
+    assert np.array_equal(count.cpu().numpy(), np.full(C, O.sample_count(N, H, W, osp), np.float32))
+    f = O.forward(x_np, gamma_np, beta_np, eps, osp)
+    b = O.backward(x_np, dy_np, gamma_np, f.mean, f.var, eps, osp)
+    tensor_close = close_f32 if dtype == "f32" else close_bf16
+    close_f32(mean.cpu().numpy(), f.mean, "mean")
+    close_f32(invstd.cpu().numpy(), f.invstd, "invstd")
+    tensor_close(np.concatenate([_to_host(t) for t in ys]), f.y, "y")
+    tensor_close(np.concatenate([_to_host(t) for t in dxs]), b.dx, "dx")
+    close_f32(sums[0].cpu().numpy(), b.dbeta, "dbeta")
+    close_f32(sums[1].cpu().numpy(), b.dgamma, "dgamma")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_statistics_from_a_fraction_of_the_ranks(dtype):
+    """Micro-BN, variant (2) of Sec. 4.3 (Batch Sampling over GPUs): only some ranks contribute statistics.
+    Three ranks, the middle one samples nothing (sampling=None): the result must be the oracle's for the whole
+    batch with a sampled set that lies in the first and the last slice only."""
+    import torch
+    from paper_1810_10962_b200 import bns
+    from helpers import quantise
+    ranks, n_local, C, H, W = 3, 6, 12, 10, 10
+    N = ranks * n_local
+    x_np = quantise(I.correlated_activations(N, C, H, W, 99), dtype)
+    dy_np = quantise(I.upstream_gradient(x_np.shape, 99), dtype)
+    gamma_np, beta_np = I.affine_parameters(C, 99)
+    gamma, beta = torch.from_numpy(gamma_np).cuda(), torch.from_numpy(beta_np).cuda()
+    eps = 1e-5
+    local = [np.array([0, 3], np.int32), None, np.array([2, 4, 5], np.int32)]
+    osp = O.Sampling.batch(np.concatenate([idx + r * n_local for r, idx in enumerate(local) if idx is not None]))
+    sps = [None if idx is None else bns.Sampling.batch(idx) for idx in local]
+    xs = [_to_device(x_np[r * n_local:(r + 1) * n_local], dtype) for r in range(ranks)]
+    dys = [_to_device(dy_np[r * n_local:(r + 1) * n_local], dtype) for r in range(ranks)]
+    gathered = torch.stack([bns.sync_local_moments(xs[r], sps[r], eps) for r in range(ranks)])
+    assert float(gathered[1].abs().max()) == 0.0                      # the silent rank: a count of zero
+    mean, invstd, count = bns.sync_merge_moments(gathered, eps)
+    ys = [bns.sync_normalize(xs[r], gamma, beta, mean, invstd) for r in range(ranks)]
+    partial = [bns.sync_backward_sums(xs[r], dys[r], gamma, mean, invstd) for r in range(ranks)]
+    sums = torch.stack([p[1] for p in partial]).sum(dim=0)
+    dxs = [bns.sync_backward_apply(xs[r], dys[r], gamma, mean, invstd, sps[r], sums, count, partial[r][0])
            for r in range(ranks)]
     torch.cuda.synchronize()
     f = O.forward(x_np, gamma_np, beta_np, eps, osp)
@@ -148,6 +188,51 @@ def test_statistics_shared_by_several_ranks_equal_one_big_batch(rule, dtype, ran
     close_f32(invstd.cpu().numpy(), f.invstd, "invstd")
     tensor_close(np.concatenate([_to_host(t) for t in ys]), f.y, "y")
     tensor_close(np.concatenate([_to_host(t) for t in dxs]), b.dx, "dx")
+    close_f32(sums[0].cpu().numpy(), b.dbeta, "dbeta")
+    close_f32(sums[1].cpu().numpy(), b.dgamma, "dgamma")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("with_dyv", [True, False])
+def test_virtual_samples_fed_to_one_rank(dtype, with_dyv):
+    """Micro-BN, variant (3) of Sec. 4.3: the virtual samples go to one rank, the others contribute nothing.
+    The result must be the oracle's VIRTUAL rule on the whole batch, dxv included."""
+    import torch
+    from paper_1810_10962_b200 import bns
+    from helpers import quantise
+    ranks, n_local, C, H, W = 2, 7, 10, 12, 12
+    N = ranks * n_local
+    x_np = quantise(I.correlated_activations(N, C, H, W, 100), dtype)
+    dy_np = quantise(I.upstream_gradient(x_np.shape, 100), dtype)
+    xv_np = I.virtual_samples(2, C, H, W, 100)
+    dyv_np = I.upstream_gradient(xv_np.shape, 100, I.TAG_DYV) if with_dyv else None
+    gamma_np, beta_np = I.affine_parameters(C, 100)
+    gamma, beta = torch.from_numpy(gamma_np).cuda(), torch.from_numpy(beta_np).cuda()
+    eps = 1e-5
+    xv = torch.from_numpy(xv_np).cuda()
+    dyv = torch.from_numpy(dyv_np).cuda() if with_dyv else None
+    sps = [bns.Sampling.virtual(xv, yv=torch.empty_like(xv), dyv=dyv, dxv=torch.empty_like(xv)), None]
+    xs = [_to_device(x_np[r * n_local:(r + 1) * n_local], dtype) for r in range(ranks)]
+    dys = [_to_device(dy_np[r * n_local:(r + 1) * n_local], dtype) for r in range(ranks)]
+    gathered = torch.stack([bns.sync_local_moments(xs[r], sps[r], eps) for r in range(ranks)])
+    mean, invstd, count = bns.sync_merge_moments(gathered, eps)
+    ys = [bns.sync_normalize(xs[r], gamma, beta, mean, invstd) for r in range(ranks)]
+    bns.sync_normalize(xv, gamma, beta, mean, invstd, y=sps[0].yv)
+    partial = [bns.sync_backward_sums(xs[r], dys[r], gamma, mean, invstd, virtual_rows=sps[r]) for r in range(ranks)]
+    sums = torch.stack([p[1] for p in partial]).sum(dim=0)
+    dxs = [bns.sync_backward_apply(xs[r], dys[r], gamma, mean, invstd, sps[r], sums, count, partial[r][0])
+           for r in range(ranks)]
+    torch.cuda.synchronize()
+    osp = O.Sampling.virtual(2)
+    f = O.forward(x_np, gamma_np, beta_np, eps, osp, xv=xv_np)
+    b = O.backward(x_np, dy_np, gamma_np, f.mean, f.var, eps, osp, xv=xv_np, dyv=dyv_np)
+    tensor_close = close_f32 if dtype == "f32" else close_bf16
+    close_f32(mean.cpu().numpy(), f.mean, "mean")
+    close_f32(invstd.cpu().numpy(), f.invstd, "invstd")
+    tensor_close(np.concatenate([_to_host(t) for t in ys]), f.y, "y")
+    close_f32(sps[0].yv.cpu().numpy(), f.yv, "yv")
+    tensor_close(np.concatenate([_to_host(t) for t in dxs]), b.dx, "dx")
+    close_f32(sps[0].dxv.cpu().numpy(), b.dxv, "dxv")
     close_f32(sums[0].cpu().numpy(), b.dbeta, "dbeta")
     close_f32(sums[1].cpu().numpy(), b.dgamma, "dgamma")
 
