@@ -435,6 +435,7 @@ bns_status clear_status(const Problem& pb, void* ws, cudaStream_t stream, unsign
 
 // ------------------------------------------------------------------------------------ launches
 bool g_pdl = true;    // ask for programmatic dependent launch (blocks may be scheduled while the previous kernel drains)
+bool g_fold_finalize = true;  // let the second backward pass finish the sums of Eq. 5 itself where it can
 bool g_l2_order = true;  // order rows so that a kernel re-reads what the previous one left in L2
 
 template <typename... KArgs, typename... Args>
@@ -754,8 +755,17 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
                                 stream, in<T>(x), in<T>(dy), out<T>(dx), gamma, mean, sink, pb.HW, set, status)));
         return last_error();
     }
-    launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
-    // pass 2: the statistics terms, on S only
+    // pass 2: the statistics terms, on S only.  Where a tile of the second pass meets few channels, its kernel
+    // finishes the sums of Eq. 5 itself (every block re-adds the partials of its channels in the same fixed
+    // order, one block per channel publishes dgamma / dbeta); otherwise a finalize launch comes first.
+    const bool has_second_pass = pb.rule != BNS_RULE_VIRTUAL || sp->dxv;
+    const int second_pass_slots = pb.rule == BNS_RULE_FEATURE ? pb.patch_plan.max_slots
+                                  : pb.rule == BNS_RULE_FULL  ? pl.max_slots
+                                                              : pv.max_slots;
+    // (not for full BN: its second pass is a stream over the whole tensor, whose many short-lived blocks would each
+    // pay the latency of re-adding the partials before their first load - measured 3 % slower)
+    const int fold = g_fold_finalize && !full && has_second_pass && second_pass_slots <= kFoldSlots ? 1 : 0;
+    if (!fold) launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
     const float inv_s = static_cast<float>(1.0 / pb.s);
     switch (pb.rule) {
     case BNS_RULE_FULL:
@@ -763,7 +773,7 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
                       (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pl.grid(), stream, in<T>(x), in<T>(dy),
                               out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, static_cast<const int*>(nullptr), 0,
                               RowOrder{g_l2_order ? RowOrder::kReversed : RowOrder::kIdentity, pl.rows, 0, 0}, pl.nchunks,
-                              pl.tiles, pb.HW, pb.P)));
+                              pl.tiles, pb.HW, pb.P, sink, fold)));
         break;
     case BNS_RULE_BATCH: {
         const int* list = nullptr;
@@ -772,7 +782,7 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
         BNS_BY_TYPE_V(pb.dtype, pv.V,
                       (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(x), in<T>(dy),
                               out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, list, pb.begin,
-                              RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P)));
+                              RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P, sink, fold)));
         break;
     }
     case BNS_RULE_FEATURE: {
@@ -782,7 +792,7 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
         const PatchPlan& pp = pb.patch_plan;
         BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, patch_fixup_kernel<T>, pp.grid(), stream, in<T>(x), in<T>(dy),
                                       out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, pb.patch, pb.N, pb.C, pb.H,
-                                      pb.W, pp.nchunks, pp.tiles, status)));
+                                      pb.W, pp.nchunks, pp.tiles, status, sink, fold)));
         break;
     }
     case BNS_RULE_VIRTUAL:
@@ -791,7 +801,7 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
                           (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(sp->xv),
                                   in<T>(sp->dyv), out<T>(sp->dxv), gamma, mean, invstd, dgamma, dbeta, inv_s,
                                   static_cast<const int*>(nullptr), 0, RowOrder{RowOrder::kIdentity, pv.rows, 0, 0},
-                                  pv.nchunks, pv.tiles, pb.HW, pb.P)));
+                                  pv.nchunks, pv.tiles, pb.HW, pb.P, sink, fold)));
         break;
     }
     return last_error();
@@ -887,7 +897,7 @@ bns_status backward_mixed_impl(const MixedProblem& mp, const bns_sampling* sp, c
         BNS_BY_TYPE_V(pr.dtype, ps.V,
                       (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, ps.grid(), stream, in<T>(x), in<T>(dy),
                               out<T>(dx), gamma, mean_s, invstd, dgamma, dbeta, w_s, list, pr.begin,
-                              RowOrder{RowOrder::kIdentity, ps.rows, 0, 0}, ps.nchunks, ps.tiles, pr.HW, pr.P)));
+                              RowOrder{RowOrder::kIdentity, ps.rows, 0, 0}, ps.nchunks, ps.tiles, pr.HW, pr.P, GradSink{}, 0)));
     } else {
         unsigned* status;
         bns_status st = clear_status(pr, ws, stream, &status);
@@ -895,7 +905,7 @@ bns_status backward_mixed_impl(const MixedProblem& mp, const bns_sampling* sp, c
         const PatchPlan& pp = pr.patch_plan;
         BNS_BY_TYPE(pr.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, patch_fixup_kernel<T>, pp.grid(), stream, in<T>(x), in<T>(dy),
                                       out<T>(dx), gamma, mean_s, invstd, dgamma, dbeta, w_s, pr.patch, pr.N, pr.C, pr.H,
-                                      pr.W, pp.nchunks, pp.tiles, status)));
+                                      pr.W, pp.nchunks, pp.tiles, status, GradSink{}, 0)));
     }
     // and on the virtual samples: share mix, spread over s_v elements, about the virtual mean
     if (sp->dxv) {
@@ -904,7 +914,7 @@ bns_status backward_mixed_impl(const MixedProblem& mp, const bns_sampling* sp, c
                       (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pq.grid(), stream, in<T>(sp->xv),
                               in<T>(sp->dyv), out<T>(sp->dxv), gamma, mean_v, invstd, dgamma, dbeta, w_v,
                               static_cast<const int*>(nullptr), 0, RowOrder{RowOrder::kIdentity, pq.rows, 0, 0},
-                              pq.nchunks, pq.tiles, pr.HW, pr.P)));
+                              pq.nchunks, pq.tiles, pr.HW, pr.P, GradSink{}, 0)));
     }
     return last_error();
 }
@@ -1359,6 +1369,7 @@ int bns_set_tuning(const char* name, int value) {
                  {"slab_max_mb", &g_slab_max_mb, nullptr, false},
                  {"slab_cluster_max", &g_slab_cluster_max, nullptr, false},
                  {"per_channel_min_hw", &g_per_channel_min_hw, nullptr, false},
+                 {"fold_finalize", nullptr, &g_fold_finalize, false},
                  {"pdl", nullptr, &g_pdl, false},
                  {"l2_order", nullptr, &g_l2_order, false}};
     for (const Knob& k : knobs) {
@@ -1603,7 +1614,7 @@ bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const 
         BNS_BY_TYPE_V(pb.dtype, pl.V,
                       (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pl.grid(), stream, in<T>(x), in<T>(dy),
                               out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, static_cast<const int*>(nullptr), 0,
-                              RowOrder{RowOrder::kIdentity, pl.rows, 0, 0}, pl.nchunks, pl.tiles, pb.HW, pb.P)));
+                              RowOrder{RowOrder::kIdentity, pl.rows, 0, 0}, pl.nchunks, pl.tiles, pb.HW, pb.P, GradSink{}, 0)));
     } else if (pb.rule == BNS_RULE_BATCH) {
         const int* list = nullptr;
         st = stage_list(pb, sampling, workspace, stream, &list);
@@ -1611,7 +1622,7 @@ bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const 
         BNS_BY_TYPE_V(pb.dtype, pv.V,
                       (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(x), in<T>(dy),
                               out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, list, pb.begin,
-                              RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P)));
+                              RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks, pv.tiles, pb.HW, pb.P, GradSink{}, 0)));
     } else if (pb.rule == BNS_RULE_FEATURE) {
         unsigned* status;
         st = clear_status(pb, workspace, stream, &status);
@@ -1619,14 +1630,14 @@ bns_status bns_sync_backward_apply(const bns_shape* shape, const void* x, const 
         const PatchPlan& pp = pb.patch_plan;
         BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, patch_fixup_kernel<T>, pp.grid(), stream, in<T>(x), in<T>(dy),
                                       out<T>(dx), gamma, mean, invstd, dgamma, dbeta, inv_s, pb.patch, pb.N, pb.C, pb.H,
-                                      pb.W, pp.nchunks, pp.tiles, status)));
+                                      pb.W, pp.nchunks, pp.tiles, status, GradSink{}, 0)));
     } else if (sampling->dxv) {
         // the virtual samples that this rank fed into the statistics: every one of them takes the upper branch
         BNS_BY_TYPE_V(sampling->xv_dtype, pv.V,
                       (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(sampling->xv),
                               in<T>(sampling->dyv), out<T>(sampling->dxv), gamma, mean, invstd, dgamma, dbeta, inv_s,
                               static_cast<const int*>(nullptr), 0, RowOrder{RowOrder::kIdentity, pv.rows, 0, 0}, pv.nchunks,
-                              pv.tiles, pb.HW, pb.P)));
+                              pv.tiles, pb.HW, pb.P, GradSink{}, 0)));
     }
     return last_error();
 }

@@ -343,7 +343,8 @@ struct GradSink {
     float* dbeta;
 };
 
-__device__ __forceinline__ void warp_finish_grads(const GradSink& G, int c, int HW, int lane) {
+// All partial sums of channel c, added in a fixed order by one warp; lane 0 returns (dgamma, dbeta).
+__device__ __forceinline__ float2 warp_sum_grads(const GradSink& G, int c, int HW, int lane) {
     float sum_dy = 0.f, sum_dyxc = 0.f;
     for (int pass = 0; pass < 2; ++pass) {
         const float2* src = pass ? G.partials_v : G.partials;
@@ -366,10 +367,40 @@ __device__ __forceinline__ void warp_finish_grads(const GradSink& G, int c, int 
         sum_dy += __shfl_down_sync(0xffffffffu, sum_dy, d);
         sum_dyxc += __shfl_down_sync(0xffffffffu, sum_dyxc, d);
     }
+    return make_float2(sum_dyxc * G.invstd[c], sum_dy);
+}
+
+__device__ __forceinline__ void warp_finish_grads(const GradSink& G, int c, int HW, int lane) {
+    const float2 g = warp_sum_grads(G, c, HW, lane);
     if (lane == 0) {
-        G.dbeta[c] = sum_dy;
-        G.dgamma[c] = sum_dyxc * G.invstd[c];
+        G.dgamma[c] = g.x;
+        G.dbeta[c] = g.y;
     }
+}
+
+// The fix-up kernels can finish the sums themselves instead of reading dgamma / dbeta from a finalize
+// launch: every block adds up, in the same fixed order, the partials of the (few) channels its tile
+// meets, and the one block that holds a channel's first position in the first row chunk publishes them.
+// s_grad[slot] = (dgamma, dbeta) of channel c_first + slot; ends with a block barrier.
+constexpr int kFoldSlots = 32;  // most channels per tile for which a fix-up kernel finishes the sums itself
+
+__device__ __forceinline__ void block_finish_grads(const GradSink& G, int c_first, int nslots, int HW, bool first_chunk,
+                                                   unsigned tile, unsigned positions_per_tile, int positions_per_channel,
+                                                   float2* s_grad) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int slot = warp; slot < nslots; slot += kThreads / 32) {
+        const int c = c_first + slot;
+        const float2 g = warp_sum_grads(G, c, HW, lane);
+        if (lane == 0) {
+            s_grad[slot] = g;
+            const unsigned home = static_cast<unsigned>(c) * static_cast<unsigned>(positions_per_channel) / positions_per_tile;
+            if (first_chunk && home == tile) {
+                G.dgamma[c] = g.x;
+                G.dbeta[c] = g.y;
+            }
+        }
+    }
+    __syncthreads();
 }
 
 // Folds the per-position moments of a block's tile (shared memory, one entry per position, every
@@ -927,25 +958,33 @@ __device__ __forceinline__ FixCoef fix_coef(float gamma, float mean, float invst
 }
 
 // Rows given by `list` (or begin .. begin+count-1): dx = a dy - A - Q (x - mean); dy == NULL reads as zeros.
+// With `fold` the kernel finishes the sums of Eq. 5 itself from the partials in G (see block_finish_grads)
+// and dgamma / dbeta are not read.
 template <typename T, int V>
 __global__ void __launch_bounds__(kThreads)
 col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
                  typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
                  const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
                  float inv_s, const int* __restrict__ list, int begin, RowOrder order, int nchunks, unsigned tiles,
-                 int HW, unsigned P) {
+                 int HW, unsigned P, GradSink G, int fold) {
+    __shared__ float2 s_grad[kFoldSlots];
     grid_dependency_wait();
     grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
     const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
+    const TileChannels tc(tile, kThreads * V, P, HW);
+    if (fold) block_finish_grads(G, tc.c_first, tc.nslots, HW, ck == 0, tile, kThreads * V, HW, s_grad);
     if (p >= P) return;
     FixCoef k[V];
     {
         int c[V];
         position_channels<V>(p, HW, c);
 #pragma unroll
-        for (int j = 0; j < V; ++j) k[j] = fix_coef(gamma[c[j]], mean[c[j]], invstd[c[j]], dgamma[c[j]], dbeta[c[j]], inv_s);
+        for (int j = 0; j < V; ++j) {
+            const float2 g = fold ? s_grad[c[j] - tc.c_first] : make_float2(dgamma[c[j]], dbeta[c[j]]);
+            k[j] = fix_coef(gamma[c[j]], mean[c[j]], invstd[c[j]], g.x, g.y, inv_s);
+        }
     }
     int i = ck;
     for (; i + (kUnroll - 1) * nchunks < order.rows; i += kUnroll * nchunks) {
@@ -991,16 +1030,21 @@ patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::
                    typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
                    const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
                    float inv_s, PatchRule rule, int N, int C, int H, int W, int nchunks, unsigned tiles,
-                   unsigned* status) {
+                   unsigned* status, GradSink G, int fold) {
+    __shared__ float2 s_grad[kFoldSlots];
     grid_dependency_wait();
     grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
     const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned j = tile * kThreads + threadIdx.x;
-    if (j >= static_cast<unsigned>(C) * rule.ph * rule.pw) return;
+    const int PP = rule.ph * rule.pw;
+    const TileChannels tc(tile, kThreads, static_cast<unsigned>(C) * PP, PP);  // channels of the tile's compact positions
+    if (fold) block_finish_grads(G, tc.c_first, tc.nslots, H * W, ck == 0, tile, kThreads, PP, s_grad);
+    if (j >= static_cast<unsigned>(C) * PP) return;
     const PatchThread me(j, rule, H, W);
     const size_t P = static_cast<size_t>(C) * H * W;
-    const FixCoef k = fix_coef(gamma[me.c], mean[me.c], invstd[me.c], dgamma[me.c], dbeta[me.c], inv_s);
+    const float2 grads = fold ? s_grad[me.c - tc.c_first] : make_float2(dgamma[me.c], dbeta[me.c]);
+    const FixCoef k = fix_coef(gamma[me.c], mean[me.c], invstd[me.c], grads.x, grads.y, inv_s);
     int n = ck;
     for (; n + (kUnroll - 1) * nchunks < N; n += kUnroll * nchunks) {
         size_t at[kUnroll];
@@ -1101,9 +1145,27 @@ direct_finalize_fixup_kernel(const typename T::storage* __restrict__ src, const 
                              typename T::storage* __restrict__ dst, const float* __restrict__ gamma,
                              const float* __restrict__ mean, GradSink G, int HW, SampleSet set, unsigned* status) {
     __shared__ float s_grad[2];
+    const int c = blockIdx.x;
+    // src and dy are inputs of the whole call (the kernels ahead of this one in the call only write dst and the
+    // partial sums), so the first batch of sampled elements is requested before the wait for those kernels.
+    // Not when patch locations come from device memory: reading them may raise the status flag, which the
+    // call clears just ahead of this kernel.
+    const bool early = dst && !(set.patches && set.patch.offsets);
+    size_t at[kUnroll];
+    float g[kUnroll], xv[kUnroll];
+    if (early) {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int q = threadIdx.x + u * kThreads;
+            if (q < set.s) {
+                at[u] = set.at(c, q, status);
+                g[u] = dy ? to_float<T>(dy[at[u]]) : 0.f;
+                xv[u] = to_float<T>(src[at[u]]);
+            }
+        }
+    }
     grid_dependency_wait();
     grid_dependency_launch();
-    const int c = blockIdx.x;
     if (threadIdx.x < 32) warp_finish_grads(G, c, HW, threadIdx.x);  // lane 0 writes dgamma[c], dbeta[c]
     __syncthreads();
     if (!dst) return;
@@ -1114,15 +1176,15 @@ direct_finalize_fixup_kernel(const typename T::storage* __restrict__ src, const 
     __syncthreads();
     const FixCoef k = fix_coef(gamma[c], mean[c], G.invstd[c], s_grad[0], s_grad[1], 1.0f / static_cast<float>(set.s));
     for (int q0 = threadIdx.x; q0 < set.s; q0 += kThreads * kUnroll) {
-        size_t at[kUnroll];
-        float g[kUnroll], xv[kUnroll];
+        if (!(early && q0 == static_cast<int>(threadIdx.x))) {
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int q = q0 + u * kThreads;
-            if (q < set.s) {
-                at[u] = set.at(c, q, status);
-                g[u] = dy ? to_float<T>(dy[at[u]]) : 0.f;
-                xv[u] = to_float<T>(src[at[u]]);
+            for (int u = 0; u < kUnroll; ++u) {
+                const int q = q0 + u * kThreads;
+                if (q < set.s) {
+                    at[u] = set.at(c, q, status);
+                    g[u] = dy ? to_float<T>(dy[at[u]]) : 0.f;
+                    xv[u] = to_float<T>(src[at[u]]);
+                }
             }
         }
 #pragma unroll
@@ -1231,11 +1293,24 @@ act_normalize_kernel(const typename T::storage* __restrict__ x, const typename T
                      typename T::storage* __restrict__ y, const float* __restrict__ gamma,
                      const float* __restrict__ beta, const float* __restrict__ mean, const float* __restrict__ invstd,
                      int rows, int nchunks, unsigned tiles, int HW, unsigned P) {
-    grid_dependency_wait();
-    grid_dependency_launch();
     const unsigned tile = blockIdx.x % tiles;
     const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
+    // x and the residual are inputs of the whole call: the first batch of rows is requested before the
+    // statistics kernels ahead of this one have finished (as in col_normalize_kernel)
+    int i = ck;
+    Vec<T, V> vx[kUnroll], vr[kUnroll];
+    if (p < P) {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (i + u * nchunks < rows) {
+                const size_t off = static_cast<size_t>(i + u * nchunks) * P + p;
+                vx[u].load(x + off);
+                if (res) vr[u].load(res + off);
+            }
+    }
+    grid_dependency_wait();
+    grid_dependency_launch();
     if (p >= P) return;
     float a[V], b[V];
     {
@@ -1247,15 +1322,7 @@ act_normalize_kernel(const typename T::storage* __restrict__ x, const typename T
             b[j] = fmaf(-mean[c[j]], a[j], beta[c[j]]);
         }
     }
-    for (int i = ck; i < rows; i += kUnroll * nchunks) {
-        Vec<T, V> vx[kUnroll], vr[kUnroll];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
-            if (i + u * nchunks < rows) {
-                const size_t off = static_cast<size_t>(i + u * nchunks) * P + p;
-                vx[u].load(x + off);
-                if (res) vr[u].load(res + off);
-            }
+    while (true) {
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u)
             if (i + u * nchunks < rows) {
@@ -1266,6 +1333,15 @@ act_normalize_kernel(const typename T::storage* __restrict__ x, const typename T
                     vx[u].set(j, fmaxf(z, 0.f));
                 }
                 vx[u].store(y + static_cast<size_t>(i + u * nchunks) * P + p);
+            }
+        i += kUnroll * nchunks;
+        if (i >= rows) break;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (i + u * nchunks < rows) {
+                const size_t off = static_cast<size_t>(i + u * nchunks) * P + p;
+                vx[u].load(x + off);
+                if (res) vr[u].load(res + off);
             }
     }
 }
@@ -1300,25 +1376,35 @@ act_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
                 b[j] = fmaf(-mu[j], a[j], beta[c[j]]);
             }
         }
-        for (int i = ck; i < rows; i += nchunks) {
-            const size_t off = static_cast<size_t>(i) * P + p;
-            Vec<T, V> vx, vg, vr;
-            vx.load(x + off);
-            vg.load(dy + off);
-            if (res) vr.load(res + off);
+        // batches of kUnroll rows, all loads of a batch in flight together; the last batch may be short
+        for (int i = ck; i < rows; i += kUnroll * nchunks) {
+            Vec<T, V> vx[kUnroll], vg[kUnroll], vr[kUnroll];
 #pragma unroll
-            for (int j = 0; j < V; ++j) {
-                const float xv = vx.get(j);
-                float z = fmaf(a[j], xv, b[j]);
-                if (res) z += vr.get(j);
-                const float g = z > 0.f ? vg.get(j) : 0.f;
-                acc_dy[j] += g;
-                acc_dyxc[j] = fmaf(g, xv - mu[j], acc_dyxc[j]);
-                vg.set(j, g);
-                vx.set(j, a[j] * g);
-            }
-            vx.store(dx + off);
-            if (dres) vg.store(dres + off);
+            for (int u = 0; u < kUnroll; ++u)
+                if (i + u * nchunks < rows) {
+                    const size_t off = static_cast<size_t>(i + u * nchunks) * P + p;
+                    vx[u].load(x + off);
+                    vg[u].load(dy + off);
+                    if (res) vr[u].load(res + off);
+                }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                if (i + u * nchunks < rows) {
+                    const size_t off = static_cast<size_t>(i + u * nchunks) * P + p;
+#pragma unroll
+                    for (int j = 0; j < V; ++j) {
+                        const float xv = vx[u].get(j);
+                        float z = fmaf(a[j], xv, b[j]);
+                        if (res) z += vr[u].get(j);
+                        const float g = z > 0.f ? vg[u].get(j) : 0.f;
+                        acc_dy[j] += g;
+                        acc_dyxc[j] = fmaf(g, xv - mu[j], acc_dyxc[j]);
+                        vg[u].set(j, g);
+                        vx[u].set(j, a[j] * g);
+                    }
+                    vx[u].store(dx + off);
+                    if (dres) vg[u].store(dres + off);
+                }
         }
     }
 #pragma unroll
