@@ -685,6 +685,15 @@ bns_status forward_impl(const Problem& pb, const bns_sampling* sp, const void* x
     bns_status st = run_statistics(pb, sp, x, eps, mean, invstd, ws, stream);
     if (st != BNS_OK) return st;
     const ColPlan& pl = pb.main_plan;
+    // The few virtual samples go first: that short kernel then runs while the blocks of the large one that
+    // follows are already being scheduled and requesting their first rows.
+    if (pb.rule == BNS_RULE_VIRTUAL && sp->yv) {
+        const ColPlan& pv = pb.stat_plan;
+        BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
+                      (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pv.grid(), stream, in<T>(sp->xv),
+                              out<T>(sp->yv), gamma, beta, mean, invstd, RowOrder{RowOrder::kIdentity, pv.rows, 0, 0},
+                              pv.nchunks, pv.tiles, pb.HW, pb.P)));
+    }
     // visit first the rows that the statistics kernel has just read: they are still in L2
     RowOrder order{RowOrder::kIdentity, pb.N, 0, 0};
     if (g_l2_order && pb.rule == BNS_RULE_FULL) order.mode = RowOrder::kReversed;
@@ -693,13 +702,6 @@ bns_status forward_impl(const Problem& pb, const bns_sampling* sp, const void* x
     BNS_BY_TYPE_V(pb.dtype, pl.V,
                   (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pl.grid(), stream, in<T>(x), out<T>(y), gamma,
                           beta, mean, invstd, order, pl.nchunks, pl.tiles, pb.HW, pb.P)));
-    if (pb.rule == BNS_RULE_VIRTUAL && sp->yv) {
-        const ColPlan& pv = pb.stat_plan;
-        BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
-                      (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pv.grid(), stream, in<T>(sp->xv),
-                              out<T>(sp->yv), gamma, beta, mean, invstd, RowOrder{RowOrder::kIdentity, pv.rows, 0, 0},
-                              pv.nchunks, pv.tiles, pb.HW, pb.P)));
-    }
     return last_error();
 }
 
