@@ -169,6 +169,18 @@ bns_status bns_update_moving_average(int C, const float* mean, const float* invs
                                      int first_iteration, float* mean_ma, float* var_ma, void* cuda_stream);
 
 /*
+ * bns_forward with the moving-average update of Eq. 8 done inside it: the thread that finishes a channel's
+ * sampled statistics also updates mean_ma[c] and var_ma[c] (Var taken directly as the biased variance of
+ * the sampled set, not recovered from invstd), so a training step needs no separate C-length launch.
+ * Same arguments, outputs and workspace as bns_forward, plus alpha, first_iteration, mean_ma, var_ma as
+ * in bns_update_moving_average.
+ */
+bns_status bns_forward_training(const bns_shape* shape, const void* x, const float* gamma, const float* beta,
+                                float eps, const bns_sampling* sampling, float alpha, int first_iteration,
+                                float* mean_ma, float* var_ma, void* y, float* mean, float* invstd,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Validation-time forward (Appendix D): Eq. 1 with E and Var replaced by the recorded moving
  * averages, y = gamma (x - mean_ma) / sqrt(var_ma + eps) + beta.  Workspace as for bns_full_bn.
  */
@@ -366,7 +378,8 @@ const char* bns_kernel_name(int kernel_kind);
 
 /* Launch-shape knobs (process-wide; change them only while no call is in flight, and recompute
  * bns_workspace_bytes afterwards).  "target_blocks" / "min_chunk": blocks per launch and least rows
- * per block of the streaming kernels (0 = a multiple of the SM count); "stat_target_blocks" / "stat_min_chunk": the same for the
+ * per block of the streaming kernels (0 = a multiple of the SM count); "full_min_chunk": least rows per block for rule FULL on tensors of
+ * 32 MiB and more; "stat_target_blocks" / "stat_min_chunk": the same for the
  * statistics kernels; "direct_max": sampled elements per channel up to which one block per channel computes the
  * statistics (and, in the backward, combines the sums and applies the statistics terms) without
  * partial sums, 0 = never; "nhwc_blocks": blocks per launch of the channels-last kernels (each block leaves one partial per

@@ -34,7 +34,7 @@ EXPORTS = [
     "bns_launch_count", "bns_launch_count_reset", "bns_profile_enable", "bns_profile_read", "bns_kernel_name",
     "bns_set_tuning", "bns_slab_plan", "bns_wait_timeouts",
     "bns_workspace_bytes_mixed", "bns_forward_mixed", "bns_backward_mixed", "bns_update_moving_average",
-    "bns_inference_forward",
+    "bns_inference_forward", "bns_forward_training",
     "bns_sync_local_moments", "bns_sync_merge_moments", "bns_sync_normalize", "bns_sync_backward_sums",
     "bns_sync_backward_apply",
     "bns_forward_relu", "bns_backward_relu",
@@ -121,6 +121,8 @@ def load():
     lib.bns_backward_mixed.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, fl, smp, vp, vp, vp, vp, sz, vp]
     lib.bns_update_moving_average.restype = ctypes.c_int
     lib.bns_update_moving_average.argtypes = [ctypes.c_int, vp, vp, fl, fl, ctypes.c_int, vp, vp, vp]
+    lib.bns_forward_training.restype = ctypes.c_int
+    lib.bns_forward_training.argtypes = [shp, vp, vp, vp, fl, smp, fl, ctypes.c_int, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.bns_inference_forward.restype = ctypes.c_int
     lib.bns_inference_forward.argtypes = [shp, vp, vp, vp, fl, vp, vp, vp, vp, sz, vp]
     lib.bns_sync_local_moments.restype = ctypes.c_int
@@ -319,6 +321,24 @@ def forward(x, gamma, beta, eps, sampling: Sampling, y=None, mean=None, invstd=N
     st = load().bns_forward(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), ctypes.byref(sp),
                             _like(y, x, "y"), _vec(mean, C), _vec(invstd, C), wp, wn, _stream())
     _check(st, "bns_forward")
+    return y, mean, invstd
+
+
+def forward_training(x, gamma, beta, eps, sampling: Sampling, alpha, first_iteration, mean_ma, var_ma, y=None,
+                     workspace=None):
+    """bns_forward_training: bns_forward that also updates the moving averages of Eq. 8 in place.
+    Returns (y, mean, invstd)."""
+    _check_virtual(x, sampling)
+    sh = _shape(x)
+    sp = sampling._c(sh)
+    C = x.shape[1]
+    y = torch.empty_like(x) if y is None else y
+    mean, invstd = (torch.empty(C, dtype=torch.float32, device=x.device) for _ in range(2))
+    ws, wp, wn = _workspace(x, sampling, workspace)
+    st = load().bns_forward_training(ctypes.byref(sh), _dev(x), _vec(gamma, C), _vec(beta, C), float(eps), ctypes.byref(sp),
+                                     float(alpha), 1 if first_iteration else 0, _vec(mean_ma, C), _vec(var_ma, C),
+                                     _like(y, x, "y"), _vec(mean, C), _vec(invstd, C), wp, wn, _stream())
+    _check(st, "bns_forward_training")
     return y, mean, invstd
 
 

@@ -302,6 +302,21 @@ struct PartialLayout {
     }
 };
 
+// Eq. 8: the moving averages of E and Var that validation uses, updated by whichever thread finishes a
+// channel's statistics (X_ma = X at the first iteration, alpha X + (1 - alpha) X_ma afterwards).  Inactive
+// when mean_ma is NULL.
+struct MovingAverage {
+    float alpha;
+    int first;
+    float* mean_ma;
+    float* var_ma;
+    __device__ __forceinline__ void update(int c, float mean, float var) const {
+        if (!mean_ma) return;
+        mean_ma[c] = first ? mean : alpha * mean + (1.0f - alpha) * mean_ma[c];
+        var_ma[c] = first ? var : alpha * var + (1.0f - alpha) * var_ma[c];
+    }
+};
+
 // Statistics: where the partial moments are and where the finished mean / invstd go.
 struct StatsSink {
     float4* partials;
@@ -309,6 +324,7 @@ struct StatsSink {
     float inv_s, eps;
     float* mean;
     float* invstd;
+    MovingAverage ma;
 };
 
 // All partial moments of channel c, merged in a fixed order by one warp; mean / invstd written by lane 0.
@@ -328,6 +344,7 @@ __device__ __forceinline__ void warp_finish_stats(const StatsSink& S, int c, int
     if (lane == 0) {
         S.mean[c] = acc.mean;
         S.invstd[c] = 1.0f / sqrtf(acc.m2 * S.inv_s + S.eps);
+        S.ma.update(c, acc.mean, acc.m2 * S.inv_s);
     }
 }
 
@@ -1100,7 +1117,7 @@ struct SampleSet {
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 direct_moments_kernel(const typename T::storage* __restrict__ src, SampleSet set, float eps, float* __restrict__ mean,
-                      float* __restrict__ invstd, unsigned* status) {
+                      float* __restrict__ invstd, unsigned* status, MovingAverage ma) {
     __shared__ Moments s_warp[kThreads / 32];
     grid_dependency_wait();
     grid_dependency_launch();
@@ -1132,6 +1149,7 @@ direct_moments_kernel(const typename T::storage* __restrict__ src, SampleSet set
         for (int w = 1; w < kThreads / 32; ++w) acc = merge(acc, s_warp[w]);
         mean[c] = acc.mean;
         invstd[c] = 1.0f / sqrtf(acc.m2 / static_cast<float>(set.s) + eps);
+        ma.update(c, acc.mean, acc.m2 / static_cast<float>(set.s));
     }
 }
 

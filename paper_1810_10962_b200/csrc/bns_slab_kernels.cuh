@@ -372,7 +372,7 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 slab_forward_kernel(const typename T::storage* __restrict__ x, typename T::storage* __restrict__ y,
                     const float* __restrict__ gamma, const float* __restrict__ beta, float eps, SlabGeom geo, SlabSel sel,
-                    float* __restrict__ mean, float* __restrict__ invstd, unsigned* status) {
+                    float* __restrict__ mean, float* __restrict__ invstd, unsigned* status, MovingAverage ma) {
     using S = typename T::storage;
     constexpr int V = 16 / sizeof(S);
     extern __shared__ __align__(128) unsigned char smem[];
@@ -533,6 +533,7 @@ slab_forward_kernel(const typename T::storage* __restrict__ x, typename T::stora
         if (rank == 0) {
             mean[c0 + threadIdx.x] = all.mean;
             invstd[c0 + threadIdx.x] = is;
+            ma.update(c0 + threadIdx.x, all.mean, all.m2 * sel.inv_s);
         }
     }
     __syncthreads();

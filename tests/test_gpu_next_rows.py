@@ -102,6 +102,38 @@ def test_moving_average_and_inference_forward():
         (close_f32 if dtype == "f32" else close_bf16)(_to_host(y), want, f"inference y {dtype}")
 
 
+@pytest.mark.parametrize("dims,rule,kw", [
+    ((48, 24, 20, 20), "batch", dict(k=24)),                     # large sampled set: partial sums + finalize
+    ((48, 24, 20, 20), "feature", dict(ph=2, pw=2)),             # small sampled set: one block per channel
+    ((32, 16, 8, 8), "full", dict()),                            # small tensor, full BN: the on-chip kernel
+    ((16, 8, 14, 14), "virtual", dict(nv=2, with_dyv=False)),
+])
+def test_forward_with_the_moving_average_folded_in(dims, rule, kw):
+    """bns_forward_training over three iterations against the oracle's forward + Eq. 8, through each way the
+    library finishes its statistics."""
+    import torch
+    from paper_1810_10962_b200 import bns
+    C = dims[1]
+    alpha = 0.7
+    mean_ma, var_ma = torch.zeros(C, device="cuda"), torch.zeros(C, device="cuda")
+    o_mean = o_var = None
+    for it in range(3):
+        case = make_case(*dims, rule, seed=970 + it, **kw)
+        x = _to_device(case.x, "f32")
+        gamma, beta = torch.from_numpy(case.gamma).cuda(), torch.from_numpy(case.beta).cuda()
+        sp = gpu_sampling(case)
+        y, mean, invstd = bns.forward_training(x, gamma, beta, case.eps, sp, alpha, it == 0, mean_ma, var_ma)
+        f = O.forward(case.x, case.gamma, case.beta, case.eps, case.oracle_sampling(), xv=case.xv)
+        o_mean = O.moving_average(f.mean, o_mean, alpha, it == 0)
+        o_var = O.moving_average(f.var, o_var, alpha, it == 0)
+        torch.cuda.synchronize()
+        close_f32(_to_host(y), f.y, "y")
+        close_f32(mean.cpu().numpy(), f.mean, "mean")
+        close_f32(invstd.cpu().numpy(), f.invstd, "invstd")
+        close_f32(mean_ma.cpu().numpy(), o_mean, f"mean_ma after iteration {it}")
+        close_f32(var_ma.cpu().numpy(), o_var, f"var_ma after iteration {it}")
+
+
 @pytest.mark.parametrize("rule", ["batch", "feature", "full"])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("ranks", [2, 3])
