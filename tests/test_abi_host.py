@@ -115,3 +115,50 @@ def test_binding_checks_the_length_of_device_offsets():
     for mode, pairs in ((bns.OFF_PER_SAMPLE, 7), (bns.OFF_PER_SAMPLE, 8 * 16), (bns.OFF_PER_MAP, 8), (bns.OFF_PER_MAP, 127)):
         with pytest.raises(TypeError):
             bns.Sampling.feature(2, 2, offsets(pairs), mode)._c(shape)
+
+
+def _plan(N, C, H, W, dtype, sampling, backward):
+    lib = bns.load()
+    sh = bns._Shape(N, C, H, W, dtype)
+    sp = sampling._c(sh)
+    out = (ctypes.c_int32 * 6)()
+    ok = lib.bns_slab_plan(ctypes.byref(sh), ctypes.byref(sp), 1 if backward else 0, out)
+    return dict(zip(("channels", "cluster", "rows", "smem_bytes", "grid", "row_lanes"), out)) if ok else None
+
+
+def test_onchip_plans_respect_the_hardware_limits():
+    """Host logic of the one-launch path: which layers take it by default, and that every plan it makes fits
+    a thread-block cluster (at most 8 blocks, at most 227 KB of shared memory each, row segments of whole
+    16-byte units, every sample held by exactly one block)."""
+    full = bns.Sampling.full()
+    try:
+        # defaults: small tensors only, and not for small sampled sets
+        assert _plan(128, 32, 16, 16, bns.F32, full, False) is not None                    # 4 MiB
+        assert _plan(256, 256, 14, 14, bns.BF16, full, False) is None                      # 24.5 MiB
+        assert _plan(128, 32, 16, 16, bns.F32, bns.Sampling.feature(4, 4, np.array([0, 0])), True) is None
+        assert _plan(8, 16, 8, 8, bns.F32, bns.Sampling.batch(np.array([1, 5], np.int32)), False) is None
+        bns.set_tuning("slab_max_mb", 1 << 20)
+        bns.set_tuning("slab_small_sets", 1)
+        rng = np.random.default_rng(5)
+        seen = 0
+        for _ in range(400):
+            N, C = int(rng.integers(1, 300)), int(rng.integers(1, 40)) * int(rng.choice([1, 2, 8, 16]))
+            H, W = int(rng.integers(1, 40)), int(rng.integers(1, 40))
+            dtype = int(rng.integers(0, 2))
+            eb = 4 if dtype == bns.F32 else 2
+            for backward in (False, True):
+                p = _plan(N, C, H, W, dtype, full, backward)
+                if p is None:
+                    continue
+                seen += 1
+                G, R = p["channels"], p["cluster"]
+                assert 1 <= R <= 8 and R <= N and p["smem_bytes"] <= 227 * 1024
+                assert C % G == 0 and (G * H * W * eb) % 16 == 0 and G * H * W * eb // 16 <= 256
+                assert p["rows"] == -(-N // R) and p["grid"] == (C // G) * R
+                assert p["smem_bytes"] >= (2 if backward else 1) * p["rows"] * G * H * W * eb
+        assert seen > 50
+        # a channel whose samples cannot fit eight blocks' shared memory keeps streaming
+        assert _plan(256, 64, 56, 56, bns.F32, full, True) is None
+    finally:
+        bns.set_tuning("slab_max_mb", 6)
+        bns.set_tuning("slab_small_sets", 0)
