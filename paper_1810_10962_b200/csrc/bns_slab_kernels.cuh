@@ -5,10 +5,10 @@
 // segment travels as one bulk asynchronous copy (cp.async.bulk + mbarrier).  Block r of the cluster
 // loads the segments of its share of the N samples into shared memory: the "slab".  Everything else
 // happens on the resident copy:
-//   forward   statistics of the sampled set (two passes over shared memory: local mean, then squared
-//             deviations about it), combined across the cluster's blocks through distributed shared
-//             memory in rank order (Chan's merge; every block computes the same bits), then
-//             y = a x + b in place and bulk stores of the rows;
+//   forward   statistics of the sampled set (one pass over shared memory of sums shifted by a pivot that is
+//             itself a sampled value of the channel), combined across the cluster's blocks through
+//             distributed shared memory in rank order (Chan's merge; every block computes the same
+//             bits), then y = a x + b in place and bulk stores of the rows;
 //   backward  sum dy and sum dy (x - mean) over every element, combined the same way, then the final
 //             gradient of every element, sampled or not, written once (Eq. 6, both branches).
 // x (and dy) are read from HBM once and y (dx) written once: 2 and 3 tensor passes, one launch each,
