@@ -642,8 +642,12 @@ bns_status slab_backward(const Problem& pb, const bns_sampling* sp, const void* 
 }
 
 // Statistics of the rule's sampled set into mean / invstd: partial moments, then one warp per channel.
+// `virtual_out` (with gamma, beta): under the VIRTUAL rule with a small set, the kernel that takes the
+// statistics also writes the normalised virtual samples there and *virtual_done is set.
 bns_status run_statistics(const Problem& pb, const bns_sampling* sp, const void* x, float eps, float* mean,
-                          float* invstd, void* ws, cudaStream_t stream, const MovingAverage& ma = MovingAverage{}) {
+                          float* invstd, void* ws, cudaStream_t stream, const MovingAverage& ma = MovingAverage{},
+                          void* virtual_out = nullptr, const float* gamma = nullptr, const float* beta = nullptr,
+                          bool* virtual_done = nullptr) {
     if (small_sampled_set(pb)) {
         unsigned* status;
         bns_status st = clear_status(pb, ws, stream, &status);
@@ -655,7 +659,9 @@ bns_status run_statistics(const Problem& pb, const bns_sampling* sp, const void*
         const void* data = pb.rule == BNS_RULE_VIRTUAL ? sp->xv : x;
         const int dt = pb.rule == BNS_RULE_VIRTUAL ? sp->xv_dtype : pb.dtype;
         BNS_BY_TYPE(dt, (launch(BNS_KERNEL_DIRECT_MOMENTS, direct_moments_kernel<T>, static_cast<unsigned>(pb.C), stream,
-                                in<T>(data), set, eps, mean, invstd, status, ma)));
+                                in<T>(data), set, eps, mean, invstd, status, ma,
+                                out<T>(pb.rule == BNS_RULE_VIRTUAL ? virtual_out : nullptr), gamma, beta)));
+        if (virtual_done && pb.rule == BNS_RULE_VIRTUAL && virtual_out) *virtual_done = true;
         return last_error();
     }
     StatsSink sink{ws_at<float4>(ws, pb.off_stats), PartialLayout{}, static_cast<float>(1.0 / pb.s), eps, mean, invstd, ma};
@@ -690,12 +696,15 @@ bns_status forward_impl(const Problem& pb, const bns_sampling* sp, const void* x
                         float eps, void* y, float* mean, float* invstd, void* ws, cudaStream_t stream,
                         const MovingAverage& ma = MovingAverage{}) {
     if (pb.slab_fwd.ok) return slab_forward(pb, sp, x, gamma, beta, eps, y, mean, invstd, ws, stream, ma);
-    bns_status st = run_statistics(pb, sp, x, eps, mean, invstd, ws, stream, ma);
+    bool virtual_done = false;
+    bns_status st = run_statistics(pb, sp, x, eps, mean, invstd, ws, stream, ma,
+                                   pb.rule == BNS_RULE_VIRTUAL ? sp->yv : nullptr, gamma, beta, &virtual_done);
     if (st != BNS_OK) return st;
     const ColPlan& pl = pb.main_plan;
-    // The few virtual samples go first: that short kernel then runs while the blocks of the large one that
-    // follows are already being scheduled and requesting their first rows.
-    if (pb.rule == BNS_RULE_VIRTUAL && sp->yv) {
+    // The few virtual samples go first (unless the statistics kernel has normalised them already): that short
+    // kernel then runs while the blocks of the large one that follows are being scheduled and requesting
+    // their first rows.
+    if (pb.rule == BNS_RULE_VIRTUAL && sp->yv && !virtual_done) {
         const ColPlan& pv = pb.stat_plan;
         BNS_BY_TYPE_V(sp->xv_dtype, pv.V,
                       (launch(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pv.grid(), stream, in<T>(sp->xv),

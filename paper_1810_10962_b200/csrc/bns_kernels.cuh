@@ -1113,12 +1113,15 @@ struct SampleSet {
     }
 };
 
-// mean and invstd of channel blockIdx.x straight from its sampled elements.
+// mean and invstd of channel blockIdx.x straight from its sampled elements; if `out` is given, also
+// out = gamma (src - mean) invstd + beta on those elements.
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 direct_moments_kernel(const typename T::storage* __restrict__ src, SampleSet set, float eps, float* __restrict__ mean,
-                      float* __restrict__ invstd, unsigned* status, MovingAverage ma) {
+                      float* __restrict__ invstd, unsigned* status, MovingAverage ma, typename T::storage* __restrict__ out,
+                      const float* __restrict__ gamma, const float* __restrict__ beta) {
     __shared__ Moments s_warp[kThreads / 32];
+    __shared__ float2 s_affine;
     grid_dependency_wait();
     grid_dependency_launch();
     const int c = blockIdx.x;
@@ -1147,9 +1150,23 @@ direct_moments_kernel(const typename T::storage* __restrict__ src, SampleSet set
     if (threadIdx.x == 0) {
         Moments acc = s_warp[0];
         for (int w = 1; w < kThreads / 32; ++w) acc = merge(acc, s_warp[w]);
+        const float is = 1.0f / sqrtf(acc.m2 / static_cast<float>(set.s) + eps);
         mean[c] = acc.mean;
-        invstd[c] = 1.0f / sqrtf(acc.m2 / static_cast<float>(set.s) + eps);
+        invstd[c] = is;
         ma.update(c, acc.mean, acc.m2 / static_cast<float>(set.s));
+        if (out) {
+            const float a = gamma[c] * is;
+            s_affine = make_float2(a, fmaf(-acc.mean, a, beta[c]));
+        }
+    }
+    if (!out) return;
+    // the sampled elements themselves are normalised right here (the virtual samples of VDN: the block has
+    // just read them, so no separate launch has to)
+    __syncthreads();
+    const float2 k = s_affine;
+    for (int q = threadIdx.x; q < set.s; q += kThreads) {
+        const size_t at = set.at(c, q, status);
+        out[at] = from_float<T>(fmaf(k.x, to_float<T>(src[at]), k.y));
     }
 }
 
