@@ -1162,9 +1162,12 @@ bns_sampling full_rule() {
 // Helper stream and events of bns_forward_backward_host, one set per device, created on first use and
 // kept until the process ends (the only objects this library ever creates).  NULL if creation fails: the
 // call then runs on the caller's stream alone.
+constexpr int kHostChunks = 8;  // row chunks of the pipelined host-buffer call
+
 struct CopyLane {
     cudaStream_t stream = nullptr;
     cudaEvent_t forward_done = nullptr, y_done = nullptr;
+    cudaEvent_t chunk_done[2 * kHostChunks + 1] = {};  // forward chunks, backward chunks, the final fix-up
     bool tried = false;
 };
 CopyLane g_copy_lanes[64];
@@ -1180,12 +1183,146 @@ CopyLane* copy_lane() {
         bool ok = cudaStreamCreateWithFlags(&lane.stream, cudaStreamNonBlocking) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&lane.forward_done, cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&lane.y_done, cudaEventDisableTiming) == cudaSuccess;
+        for (cudaEvent_t& e : lane.chunk_done) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
         if (!ok) {
             cudaGetLastError();
             lane.stream = nullptr;
         }
     }
     return lane.stream ? &lane : nullptr;
+}
+
+// Device buffers of bns_forward_backward_host inside the caller's arena.
+struct HostArena {
+    void *d_x, *d_dy, *d_y, *d_dx, *ws;
+    float *d_gamma, *d_beta, *d_mean, *d_invstd, *d_dgamma, *d_dbeta, *d_chunk_grads;
+    size_t tensor_bytes, vector_bytes;
+};
+
+bool g_host_pipeline = true;  // overlap the two directions of the link by row chunks where the rule allows it
+
+// The pipelined form of the host-buffer call.  Both directions of the link work at once for most of the
+// call: what the statistics need goes up first (the sampled samples, or the patches of every map as one
+// strided copy), then x goes up in row chunks while the normalised chunks of y already travel down; dy goes
+// up in row chunks while backward pass 1 runs per chunk and the chunks of dx (correct everywhere but on the
+// sampled set) travel down; last, the sums of the chunks are added, the sampled elements get their
+// statistics terms, and only they are sent again.  One cudaMemcpyAsync (or cudaMemcpy3DAsync) per piece.
+// Returns false, having enqueued nothing, when the rule or the shape does not allow it.
+bool host_pipelined(const Problem& pb, const bns_sampling* sp, const void* x, const void* dy, const float* gamma,
+                    const float* beta, float eps, void* y, void* dx, float* mean, float* invstd, float* dgamma,
+                    float* dbeta, const HostArena& A, CopyLane* lane, cudaStream_t stream, bns_status* result) {
+    const bool batch = pb.rule == BNS_RULE_BATCH && pb.contiguous;
+    const bool feature = pb.rule == BNS_RULE_FEATURE && !pb.patch.offsets;
+    if (!g_host_pipeline || !lane || !(batch || feature) || pb.N < 4 * kHostChunks) return false;
+    const int eb = elem_bytes(pb.dtype);
+    const size_t row_bytes = static_cast<size_t>(pb.P) * eb;
+    auto at = [&](const void* p, int row) { return static_cast<const char*>(p) + static_cast<size_t>(row) * row_bytes; };
+    auto at_mut = [&](void* p, int row) { return static_cast<char*>(p) + static_cast<size_t>(row) * row_bytes; };
+    bool ok = true;
+    // rows [r0, r0+rows) of a tensor over the link, leaving out the sampled samples of Batch Sampling (they
+    // travel separately: up before everything else, down after the fix-up)
+    auto copy_rows = [&](void* dst, const void* src, int r0, int rows, cudaMemcpyKind kind, cudaStream_t s) {
+        const int skip_lo = batch ? pb.begin : 0, skip_hi = batch ? pb.begin + pb.count : 0;
+        const int a0 = r0, a1 = std::min(r0 + rows, std::max(r0, skip_lo));      // before the sampled samples
+        const int b0 = std::max(r0, std::min(r0 + rows, skip_hi)), b1 = r0 + rows;  // after them
+        if (a1 > a0)
+            ok &= cudaMemcpyAsync(at_mut(dst, a0), at(src, a0), (a1 - a0) * row_bytes, kind, s) == cudaSuccess;
+        if (b1 > b0)
+            ok &= cudaMemcpyAsync(at_mut(dst, b0), at(src, b0), (b1 - b0) * row_bytes, kind, s) == cudaSuccess;
+    };
+    auto copy_patches = [&](void* dst, const void* src, cudaMemcpyKind kind, cudaStream_t s) {
+        cudaMemcpy3DParms p = {};
+        const size_t pitch = static_cast<size_t>(pb.W) * eb;
+        p.srcPtr = make_cudaPitchedPtr(const_cast<void*>(src), pitch, pitch, pb.H);
+        p.dstPtr = make_cudaPitchedPtr(dst, pitch, pitch, pb.H);
+        p.srcPos = p.dstPos = make_cudaPos(static_cast<size_t>(pb.patch.ow) * eb, pb.patch.oh, 0);
+        p.extent = make_cudaExtent(static_cast<size_t>(pb.patch.pw) * eb, pb.patch.ph, static_cast<size_t>(pb.N) * pb.C);
+        p.kind = kind;
+        ok &= cudaMemcpy3DAsync(&p, s) == cudaSuccess;
+    };
+    ok &= cudaMemcpyAsync(A.d_gamma, gamma, A.vector_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(A.d_beta, beta, A.vector_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    // ---- forward: the sampled set first, statistics, then chunks up / normalise / chunks down
+    if (batch)
+        ok &= cudaMemcpyAsync(at_mut(A.d_x, pb.begin), at(x, pb.begin), pb.count * row_bytes, cudaMemcpyHostToDevice, stream) ==
+              cudaSuccess;
+    else
+        copy_patches(A.d_x, x, cudaMemcpyHostToDevice, stream);
+    if (!ok) {
+        *result = BNS_ERR_CUDA;
+        return true;
+    }
+    bns_status st = run_statistics(pb, sp, A.d_x, eps, A.d_mean, A.d_invstd, A.ws, stream);
+    if (st != BNS_OK) {
+        *result = st;
+        return true;
+    }
+    for (int i = 0; i < kHostChunks; ++i) {
+        const int r0 = static_cast<int>(static_cast<long long>(i) * pb.N / kHostChunks);
+        const int rows = static_cast<int>(static_cast<long long>(i + 1) * pb.N / kHostChunks) - r0;
+        copy_rows(A.d_x, x, r0, rows, cudaMemcpyHostToDevice, stream);
+        const ColPlan pl = plan_col(pb.P, pb.HW, pb.C, rows, eb);
+        BNS_BY_TYPE_V(pb.dtype, pl.V,
+                      (launch_after_predecessor(BNS_KERNEL_NORMALIZE, col_normalize_kernel<T, V>, pl.grid(), stream,
+                                                in<T>(at(A.d_x, r0)), out<T>(at_mut(A.d_y, r0)), A.d_gamma, A.d_beta, A.d_mean,
+                                                A.d_invstd, RowOrder{RowOrder::kIdentity, rows, 0, 0}, pl.nchunks, pl.tiles,
+                                                pb.HW, pb.P)));
+        ok &= cudaEventRecord(lane->chunk_done[i], stream) == cudaSuccess;
+        ok &= cudaStreamWaitEvent(lane->stream, lane->chunk_done[i], 0) == cudaSuccess;
+        ok &= cudaMemcpyAsync(at_mut(y, r0), at(A.d_y, r0), rows * row_bytes, cudaMemcpyDeviceToHost, lane->stream) == cudaSuccess;
+    }
+    // ---- backward: chunks up / pass 1 per chunk / chunks of dx down
+    for (int i = 0; i < kHostChunks; ++i) {
+        const int r0 = static_cast<int>(static_cast<long long>(i) * pb.N / kHostChunks);
+        const int rows = static_cast<int>(static_cast<long long>(i + 1) * pb.N / kHostChunks) - r0;
+        ok &= cudaMemcpyAsync(at_mut(A.d_dy, r0), at(dy, r0), rows * row_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+        const ColPlan pl = plan_col(pb.P, pb.HW, pb.C, rows, eb);
+        float* grads = A.d_chunk_grads + static_cast<size_t>(i) * 2 * pb.C;
+        GradSink sink{ws_at<float2>(A.ws, pb.off_bwd), pl.layout(), nullptr, pl.layout(), A.d_invstd, grads, grads + pb.C};
+        BNS_BY_TYPE_V(pb.dtype, pl.V,
+                      (launch_after_predecessor(BNS_KERNEL_BWD_REDUCE, bwd_reduce_variant<T, V, true>(pb.HW), pl.grid(), stream,
+                                                in<T>(at(A.d_x, r0)), in<T>(at(A.d_dy, r0)), out<T>(at_mut(A.d_dx, r0)), A.d_gamma,
+                                                A.d_mean, A.d_invstd, RowOrder{RowOrder::kIdentity, rows, 0, 0}, pl.nchunks,
+                                                pl.tiles, pb.HW, pb.P, false, sink)));
+        launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
+        ok &= cudaEventRecord(lane->chunk_done[kHostChunks + i], stream) == cudaSuccess;
+        ok &= cudaStreamWaitEvent(lane->stream, lane->chunk_done[kHostChunks + i], 0) == cudaSuccess;
+        copy_rows(dx, A.d_dx, r0, rows, cudaMemcpyDeviceToHost, lane->stream);
+    }
+    // ---- the sums of all chunks, the statistics terms on the sampled set, and that set once more down the link
+    launch(BNS_KERNEL_VECTOR, sum_chunk_grads_kernel, per_channel_grid(pb.C), stream,
+           static_cast<const float*>(A.d_chunk_grads), kHostChunks, pb.C, A.d_dgamma, A.d_dbeta);
+    const float inv_s = static_cast<float>(1.0 / pb.s);
+    if (batch) {
+        const ColPlan& pv = pb.stat_plan;
+        BNS_BY_TYPE_V(pb.dtype, pv.V,
+                      (launch(BNS_KERNEL_COL_FIXUP, col_fixup_kernel<T, V>, pv.grid(), stream, in<T>(A.d_x), in<T>(A.d_dy),
+                              out<T>(A.d_dx), A.d_gamma, A.d_mean, A.d_invstd, A.d_dgamma, A.d_dbeta, inv_s,
+                              static_cast<const int*>(nullptr), pb.begin, RowOrder{RowOrder::kIdentity, pv.rows, 0, 0},
+                              pv.nchunks, pv.tiles, pb.HW, pb.P, GradSink{}, 0)));
+    } else {
+        const PatchPlan& pp = pb.patch_plan;
+        BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, patch_fixup_kernel<T>, pp.grid(), stream, in<T>(A.d_x),
+                                      in<T>(A.d_dy), out<T>(A.d_dx), A.d_gamma, A.d_mean, A.d_invstd, A.d_dgamma, A.d_dbeta,
+                                      inv_s, pb.patch, pb.N, pb.C, pb.H, pb.W, pp.nchunks, pp.tiles,
+                                      static_cast<unsigned*>(nullptr), GradSink{}, 0)));
+    }
+    ok &= cudaEventRecord(lane->chunk_done[2 * kHostChunks], stream) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(lane->stream, lane->chunk_done[2 * kHostChunks], 0) == cudaSuccess;
+    if (batch)
+        ok &= cudaMemcpyAsync(at_mut(dx, pb.begin), at(A.d_dx, pb.begin), pb.count * row_bytes, cudaMemcpyDeviceToHost,
+                              lane->stream) == cudaSuccess;
+    else
+        copy_patches(dx, A.d_dx, cudaMemcpyDeviceToHost, lane->stream);
+    ok &= cudaEventRecord(lane->y_done, lane->stream) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(stream, lane->y_done, 0) == cudaSuccess;  // the helper joins the caller's stream
+    ok &= cudaMemcpyAsync(mean, A.d_mean, A.vector_bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(invstd, A.d_invstd, A.vector_bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(dgamma, A.d_dgamma, A.vector_bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(dbeta, A.d_dbeta, A.vector_bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    const bns_status launches = last_error();
+    *result = !ok ? BNS_ERR_CUDA : launches;
+    return true;
 }
 
 // ======================================================================================== C ABI
@@ -1237,7 +1374,7 @@ size_t bns_host_arena_bytes(const bns_shape* shape, const bns_sampling* sampling
     if (make_problem(shape, sampling, pb) != BNS_OK) return 0;
     const size_t tensor = align_up(pb.elems * elem_bytes(pb.dtype));
     const size_t vec = align_up(static_cast<size_t>(pb.C) * sizeof(float));
-    return 4 * tensor + 6 * vec + align_up(pb.total);
+    return 4 * tensor + 6 * vec + align_up(pb.total) + 2 * kHostChunks * vec;
 }
 
 bns_status bns_forward_backward_host(const bns_shape* shape, const void* x, const void* dy, const float* gamma,
@@ -1266,6 +1403,15 @@ bns_status bns_forward_backward_host(const bns_shape* shape, const void* x, cons
     void* ws = base + 4 * tensor + 6 * vec;
     float *d_gamma = d_vec[0], *d_beta = d_vec[1], *d_mean = d_vec[2], *d_invstd = d_vec[3], *d_dgamma = d_vec[4],
           *d_dbeta = d_vec[5];
+    {
+        void* after_ws = base + 4 * tensor + 6 * vec + align_up(pb.total);
+        const HostArena A{d_x, d_dy, d_y, d_dx, ws, d_gamma, d_beta, d_mean, d_invstd, d_dgamma, d_dbeta,
+                          static_cast<float*>(after_ws), tbytes, vbytes};
+        bns_status piped = BNS_OK;
+        if (host_pipelined(pb, sampling, x, dy, gamma, beta, eps, y, dx, mean, invstd, dgamma, dbeta, A, copy_lane(), stream,
+                           &piped))
+            return piped;
+    }
     bool ok = true;
     ok &= cudaMemcpyAsync(d_x, x, tbytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
     ok &= cudaMemcpyAsync(d_gamma, gamma, vbytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
@@ -1390,6 +1536,7 @@ int bns_set_tuning(const char* name, int value) {
                  {"slab_cluster_max", &g_slab_cluster_max, nullptr, false},
                  {"per_channel_min_hw", &g_per_channel_min_hw, nullptr, false},
                  {"fold_finalize", nullptr, &g_fold_finalize, false},
+                 {"host_pipeline", nullptr, &g_host_pipeline, false},
                  {"pdl", nullptr, &g_pdl, false},
                  {"l2_order", nullptr, &g_l2_order, false}};
     for (const Knob& k : knobs) {

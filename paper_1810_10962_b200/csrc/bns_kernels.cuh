@@ -1267,6 +1267,23 @@ invstd_from_var_kernel(const float* __restrict__ var, float eps, int C, float* _
     if (c < C) invstd[c] = 1.0f / sqrtf(var[c] + eps);
 }
 
+// Adds up, in index order, the (dgamma, dbeta) vectors that n row chunks of one layer left behind
+// (chunk i at rows[i*2C .. i*2C+C) and rows[i*2C+C .. (i+1)*2C)).
+__global__ void __launch_bounds__(kThreads)
+sum_chunk_grads_kernel(const float* __restrict__ rows, int n, int C, float* __restrict__ dgamma, float* __restrict__ dbeta) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const int c = blockIdx.x * kThreads + threadIdx.x;
+    if (c >= C) return;
+    float g = 0.f, b = 0.f;
+    for (int i = 0; i < n; ++i) {
+        g += rows[static_cast<size_t>(i) * 2 * C + c];
+        b += rows[static_cast<size_t>(i) * 2 * C + C + c];
+    }
+    dgamma[c] = g;
+    dbeta[c] = b;
+}
+
 // ------------------------------------------------------------------------------------ statistics shared by several GPUs
 // A rank's sampled statistics as (count, mean, M2) rows of C floats, the form in which ranks exchange
 // them; rows 1 and 2 arrive holding mean and invstd and row 2 is turned into M2 = count (1/invstd^2 - eps).

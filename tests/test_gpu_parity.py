@@ -309,15 +309,18 @@ def test_small_patches(ph, pw, mode, dtype, dims):
     compare(case, run_gpu(case))
 
 
-@pytest.mark.parametrize("rule,kw", [("batch", dict(k=4)), ("feature", dict(ph=3, pw=3)), ("full", dict())])
+@pytest.mark.parametrize("rule,kw,N", [("batch", dict(k=4), 20), ("feature", dict(ph=3, pw=3), 20), ("full", dict(), 20),
+                                       # 32 samples and more: the two directions of the link overlap by row chunks
+                                       ("batch", dict(k=6), 45), ("batch", dict(k=33), 67), ("feature", dict(ph=3, pw=2), 45),
+                                       ("feature", dict(ph=10, pw=10), 32), ("batch", dict(k=5, contiguous=False), 40)])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_host_buffer_entry_point(rule, kw, dtype):
+def test_host_buffer_entry_point(rule, kw, N, dtype):
     """bns_forward_backward_host: pinned host tensors in, pinned host tensors out, copies on the stream."""
     import torch
     from paper_1810_10962_b200 import bns
     from helpers import run_oracle, close_f32, close_bf16, _to_host
     import bns_inputs as I
-    case = make_case(20, 12, 10, 10, rule, seed=89, dtype=dtype, **kw)
+    case = make_case(N, 12, 10, 10, rule, seed=89, dtype=dtype, **kw)
     dt = torch.float32 if dtype == "f32" else torch.bfloat16
 
     def pin(a):
