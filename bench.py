@@ -627,11 +627,14 @@ def run_ours(args):
         del dev
         torch.cuda.empty_cache()
         others = {}
+        oargs = argparse.Namespace(**vars(args))
+        oargs.steps = min(args.steps, 20)          # bounded: these are side measurements of the same run
         for name in OTHER_CONFIGS:
             olayers = workload_layers(name)
             oin = [device_inputs(l, layer_seed(name, i), torch) for i, l in enumerate(olayers)]
-            res, odev = measure_workload(torch, dist, bns, args, olayers, oin, local, world, args.seconds / 2,
+            res, odev = measure_workload(torch, dist, bns, oargs, olayers, oin, local, world, args.seconds / 2,
                                          args.seconds / 8, warm=name in ("cifar", "vdn"))
+            res["steps_per_repeat"] = oargs.steps
             res["frac_of_hbm_peak"] = round(res["value"] / peak, 4)
             res["frac_of_nominal_8TBps"] = round(res["value"] / NOMINAL_HBM_GBS, 4)
             res["layers"] = [f"{l.name}:{l.N}x{l.C}x{l.H}x{l.W}:{l.dtype}:x{l.count}" for l in olayers]
