@@ -531,6 +531,14 @@ unsigned warp_per_channel_grid(int C) { return static_cast<unsigned>((C + kThrea
 // Small sampled sets are handled by one block per channel (no partials, no finalize launch).
 bool small_sampled_set(const Problem& pb) { return pb.rule != BNS_RULE_FULL && pb.s <= static_cast<double>(g_direct_max); }
 
+// The one-block-per-channel kernels come in two depths.  With more than kUnroll elements per thread and few
+// enough channels for all blocks to be resident at the larger register count, a thread keeps kDirectUnroll
+// loads in flight: fewer dependent trips to memory (CIFAR sweep 53 -> 48 us per step).  With more channels the
+// lost occupancy costs more than that (256x512x28x28, 3x3 patches: second pass 28.6 -> 34.7 us).
+bool deep_direct(const Problem& pb, const SampleSet& set) {
+    return set.s > kUnroll * kThreads && pb.C <= 2 * sm_count();
+}
+
 SampleSet sample_set(const Problem& pb, const int* list) {
     SampleSet set{};
     set.patches = pb.rule == BNS_RULE_FEATURE;
@@ -658,9 +666,14 @@ bns_status run_statistics(const Problem& pb, const bns_sampling* sp, const void*
         const SampleSet set = sample_set(pb, list);
         const void* data = pb.rule == BNS_RULE_VIRTUAL ? sp->xv : x;
         const int dt = pb.rule == BNS_RULE_VIRTUAL ? sp->xv_dtype : pb.dtype;
-        BNS_BY_TYPE(dt, (launch(BNS_KERNEL_DIRECT_MOMENTS, direct_moments_kernel<T>, static_cast<unsigned>(pb.C), stream,
-                                in<T>(data), set, eps, mean, invstd, status, ma,
-                                out<T>(pb.rule == BNS_RULE_VIRTUAL ? virtual_out : nullptr), gamma, beta)));
+        if (deep_direct(pb, set))
+            BNS_BY_TYPE(dt, (launch(BNS_KERNEL_DIRECT_MOMENTS, direct_moments_kernel<T, kDirectUnroll>,
+                                    static_cast<unsigned>(pb.C), stream, in<T>(data), set, eps, mean, invstd, status, ma,
+                                    out<T>(pb.rule == BNS_RULE_VIRTUAL ? virtual_out : nullptr), gamma, beta)));
+        else
+            BNS_BY_TYPE(dt, (launch(BNS_KERNEL_DIRECT_MOMENTS, direct_moments_kernel<T>, static_cast<unsigned>(pb.C), stream,
+                                    in<T>(data), set, eps, mean, invstd, status, ma,
+                                    out<T>(pb.rule == BNS_RULE_VIRTUAL ? virtual_out : nullptr), gamma, beta)));
         if (virtual_done && pb.rule == BNS_RULE_VIRTUAL && virtual_out) *virtual_done = true;
         return last_error();
     }
@@ -763,11 +776,22 @@ bns_status backward_impl(const Problem& pb, const bns_sampling* sp, const void* 
         st = stage_list(pb, sp, ws, stream, &list);
         if (st != BNS_OK) return st;
         const SampleSet set = sample_set(pb, list);
-        if (pb.rule == BNS_RULE_VIRTUAL)
+        const bool deep = deep_direct(pb, set);
+        if (pb.rule == BNS_RULE_VIRTUAL && deep)
+            BNS_BY_TYPE(sp->xv_dtype,
+                        (launch(BNS_KERNEL_DIRECT_FIXUP, direct_finalize_fixup_kernel<T, kDirectUnroll>,
+                                static_cast<unsigned>(pb.C), stream, in<T>(sp->xv), in<T>(sp->dyv), out<T>(sp->dxv), gamma,
+                                mean, sink, pb.HW, set, status)));
+        else if (pb.rule == BNS_RULE_VIRTUAL)
             BNS_BY_TYPE(sp->xv_dtype,
                         (launch(BNS_KERNEL_DIRECT_FIXUP, direct_finalize_fixup_kernel<T>, static_cast<unsigned>(pb.C),
                                 stream, in<T>(sp->xv), in<T>(sp->dyv), out<T>(sp->dxv), gamma, mean, sink, pb.HW, set,
                                 status)));
+        else if (deep)
+            BNS_BY_TYPE(pb.dtype,
+                        (launch(BNS_KERNEL_DIRECT_FIXUP, direct_finalize_fixup_kernel<T, kDirectUnroll>,
+                                static_cast<unsigned>(pb.C), stream, in<T>(x), in<T>(dy), out<T>(dx), gamma, mean, sink,
+                                pb.HW, set, status)));
         else
             BNS_BY_TYPE(pb.dtype,
                         (launch(BNS_KERNEL_DIRECT_FIXUP, direct_finalize_fixup_kernel<T>, static_cast<unsigned>(pb.C),

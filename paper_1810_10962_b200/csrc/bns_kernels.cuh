@@ -1115,7 +1115,10 @@ struct SampleSet {
 
 // mean and invstd of channel blockIdx.x straight from its sampled elements; if `out` is given, also
 // out = gamma (src - mean) invstd + beta on those elements.
-template <typename T>
+constexpr int kDirectUnroll = 12;
+// U: loads a thread keeps in flight (sets beyond kUnroll elements per thread take the larger value: fewer
+// dependent round trips to memory).
+template <typename T, int U = kUnroll>
 __global__ void __launch_bounds__(kThreads)
 direct_moments_kernel(const typename T::storage* __restrict__ src, SampleSet set, float eps, float* __restrict__ mean,
                       float* __restrict__ invstd, unsigned* status, MovingAverage ma, typename T::storage* __restrict__ out,
@@ -1126,16 +1129,16 @@ direct_moments_kernel(const typename T::storage* __restrict__ src, SampleSet set
     grid_dependency_launch();
     const int c = blockIdx.x;
     float K = 0.f, s1 = 0.f, s2 = 0.f, cnt = 0.f;
-    for (int q0 = threadIdx.x; q0 < set.s; q0 += kThreads * kUnroll) {
-        float v[kUnroll];
+    for (int q0 = threadIdx.x; q0 < set.s; q0 += kThreads * U) {
+        float v[U];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < U; ++u) {
             const int q = q0 + u * kThreads;
             if (q < set.s) v[u] = to_float<T>(src[set.at(c, q, status)]);
         }
         if (cnt == 0.f) K = v[0];  // pivot: the thread's first value
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < U; ++u) {
             if (q0 + u * kThreads < set.s) {
                 float d = v[u] - K;
                 s1 += d;
@@ -1174,7 +1177,7 @@ direct_moments_kernel(const typename T::storage* __restrict__ src, SampleSet set
 // kernel would), publishes dgamma / dbeta, and rewrites the gradient of the channel's sampled elements
 // with the statistics terms: dst = a dy - A - Q (src - mean).  dy == NULL reads as zeros; dst == NULL
 // skips the rewrite.
-template <typename T>
+template <typename T, int U = kUnroll>
 __global__ void __launch_bounds__(kThreads)
 direct_finalize_fixup_kernel(const typename T::storage* __restrict__ src, const typename T::storage* __restrict__ dy,
                              typename T::storage* __restrict__ dst, const float* __restrict__ gamma,
@@ -1186,11 +1189,11 @@ direct_finalize_fixup_kernel(const typename T::storage* __restrict__ src, const 
     // Not when patch locations come from device memory: reading them may raise the status flag, which the
     // call clears just ahead of this kernel.
     const bool early = dst && !(set.patches && set.patch.offsets);
-    size_t at[kUnroll];
-    float g[kUnroll], xv[kUnroll];
+    size_t at[U];
+    float g[U], xv[U];
     if (early) {
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < U; ++u) {
             const int q = threadIdx.x + u * kThreads;
             if (q < set.s) {
                 at[u] = set.at(c, q, status);
@@ -1199,21 +1202,26 @@ direct_finalize_fixup_kernel(const typename T::storage* __restrict__ src, const 
             }
         }
     }
+    // gamma, mean and invstd are inputs of the call as well
+    const float scale = gamma[c], mu = mean[c], is = G.invstd[c];
     grid_dependency_wait();
     grid_dependency_launch();
-    if (threadIdx.x < 32) warp_finish_grads(G, c, HW, threadIdx.x);  // lane 0 writes dgamma[c], dbeta[c]
-    __syncthreads();
-    if (!dst) return;
-    if (threadIdx.x == 0) {
-        s_grad[0] = G.dgamma[c];  // written by this thread just above
-        s_grad[1] = G.dbeta[c];
+    if (threadIdx.x < 32) {
+        const float2 grads = warp_sum_grads(G, c, HW, threadIdx.x);
+        if (threadIdx.x == 0) {
+            G.dgamma[c] = grads.x;
+            G.dbeta[c] = grads.y;
+            s_grad[0] = grads.x;
+            s_grad[1] = grads.y;
+        }
     }
+    if (!dst) return;
     __syncthreads();
-    const FixCoef k = fix_coef(gamma[c], mean[c], G.invstd[c], s_grad[0], s_grad[1], 1.0f / static_cast<float>(set.s));
-    for (int q0 = threadIdx.x; q0 < set.s; q0 += kThreads * kUnroll) {
+    const FixCoef k = fix_coef(scale, mu, is, s_grad[0], s_grad[1], 1.0f / static_cast<float>(set.s));
+    for (int q0 = threadIdx.x; q0 < set.s; q0 += kThreads * U) {
         if (!(early && q0 == static_cast<int>(threadIdx.x))) {
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
+            for (int u = 0; u < U; ++u) {
                 const int q = q0 + u * kThreads;
                 if (q < set.s) {
                     at[u] = set.at(c, q, status);
@@ -1223,7 +1231,7 @@ direct_finalize_fixup_kernel(const typename T::storage* __restrict__ src, const 
             }
         }
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
+        for (int u = 0; u < U; ++u)
             if (q0 + u * kThreads < set.s) dst[at[u]] = from_float<T>(fmaf(k.a, g[u], -k.A) - k.Q * (xv[u] - k.mu));
     }
 }
