@@ -1870,7 +1870,8 @@ bns_status bns_forward_relu(const bns_shape* shape, const void* x, const void* r
     const ColPlan& pl = pb.main_plan;
     BNS_BY_TYPE_V(pb.dtype, pl.V,
                   (launch(BNS_KERNEL_NORMALIZE, act_normalize_kernel<T, V>, pl.grid(), stream, in<T>(x), in<T>(residual),
-                          out<T>(y), gamma, beta, mean, invstd, pl.rows, pl.nchunks, pl.tiles, pb.HW, pb.P)));
+                          out<T>(y), gamma, beta, mean, invstd, RowOrder{RowOrder::kIdentity, pl.rows, 0, 0}, pl.nchunks,
+                          pl.tiles, pb.HW, pb.P)));
     return last_error();
 }
 
@@ -1893,9 +1894,14 @@ bns_status bns_backward_relu(const bns_shape* shape, const void* x, const void* 
     GradSink sink{ws_at<float2>(workspace, pb.off_bwd), pl.layout(), nullptr, pl.layout(), invstd, dgamma, dbeta};
     BNS_BY_TYPE_V(pb.dtype, pl.V,
                   (launch(BNS_KERNEL_BWD_REDUCE, act_bwd_reduce_kernel<T, V>, pl.grid(), stream, in<T>(x), in<T>(residual),
-                          in<T>(dy), out<T>(dx), out<T>(dresidual), gamma, beta, mean, invstd, pl.rows, pl.nchunks,
-                          pl.tiles, pb.HW, pb.P, sink)));
-    launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
+                          in<T>(dy), out<T>(dx), out<T>(dresidual), gamma, beta, mean, invstd,
+                          RowOrder{RowOrder::kIdentity, pl.rows, 0, 0}, pl.nchunks, pl.tiles, pb.HW, pb.P, sink)));
+    // the second pass finishes the sums of Eq. 5 itself where its tiles meet few channels (as in backward_impl)
+    const int second_pass_slots = pb.rule == BNS_RULE_FEATURE ? pb.patch_plan.max_slots
+                                  : pb.rule == BNS_RULE_FULL  ? pl.max_slots
+                                                              : pv.max_slots;
+    const int fold = g_fold_finalize && pb.rule != BNS_RULE_FULL && second_pass_slots <= kFoldSlots ? 1 : 0;
+    if (!fold) launch(BNS_KERNEL_FINALIZE_BWD, finalize_bwd_kernel, warp_per_channel_grid(pb.C), stream, sink, pb.C, pb.HW);
     const float inv_s = static_cast<float>(1.0 / pb.s);
     if (pb.rule == BNS_RULE_FEATURE) {
         unsigned* status;
@@ -1904,7 +1910,8 @@ bns_status bns_backward_relu(const bns_shape* shape, const void* x, const void* 
         const PatchPlan& pp = pb.patch_plan;
         BNS_BY_TYPE(pb.dtype, (launch(BNS_KERNEL_PATCH_FIXUP, act_patch_fixup_kernel<T>, pp.grid(), stream, in<T>(x),
                                       in<T>(residual), in<T>(dy), out<T>(dx), gamma, beta, mean, invstd, dgamma, dbeta,
-                                      inv_s, pb.patch, pb.N, pb.C, pb.H, pb.W, pp.nchunks, pp.tiles, status)));
+                                      inv_s, pb.patch, pb.N, pb.C, pb.H, pb.W, pp.nchunks, pp.tiles, status, sink,
+                                      fold)));
     } else {
         const int* list = nullptr;
         st = stage_list(pb, sampling, workspace, stream, &list);
@@ -1913,8 +1920,8 @@ bns_status bns_backward_relu(const bns_shape* shape, const void* x, const void* 
         BNS_BY_TYPE_V(pb.dtype, pf.V,
                       (launch(BNS_KERNEL_COL_FIXUP, act_col_fixup_kernel<T, V>, pf.grid(), stream, in<T>(x),
                               in<T>(residual), in<T>(dy), out<T>(dx), gamma, beta, mean, invstd, dgamma, dbeta, inv_s,
-                              list, pb.rule == BNS_RULE_BATCH ? pb.begin : 0, pf.rows, pf.nchunks, pf.tiles, pb.HW,
-                              pb.P)));
+                              list, pb.rule == BNS_RULE_BATCH ? pb.begin : 0,
+                              RowOrder{RowOrder::kIdentity, pf.rows, 0, 0}, pf.nchunks, pf.tiles, pb.HW, pb.P, sink, fold)));
     }
     return last_error();
 }

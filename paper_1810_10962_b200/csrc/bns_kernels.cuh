@@ -685,21 +685,26 @@ finalize_bwd_kernel(GradSink G, int C, int HW) {
 
 // ------------------------------------------------------------------------------------ normalise + affine
 // y = a_c x + b_c with a_c = gamma_c invstd_c and b_c = beta_c - mean_c a_c, over the rows of the chunk.
-template <typename T, int V>
-__global__ void __launch_bounds__(kThreads)
-col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::storage* __restrict__ y,
-                     const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
-                     const float* __restrict__ invstd, RowOrder order, int nchunks, unsigned tiles, int HW, unsigned P) {
+// With ACT the step that follows a BN layer in a residual network is fused in, so that the pre-activation
+// tensor is never written: y = max(0, a x + b + r), r = `res` (may be NULL).
+template <typename T, int V, bool ACT>
+__device__ __forceinline__ void normalize_rows(const typename T::storage* __restrict__ x,
+                                               const typename T::storage* __restrict__ res,
+                                               typename T::storage* __restrict__ y, const float* __restrict__ gamma,
+                                               const float* __restrict__ beta, const float* __restrict__ mean,
+                                               const float* __restrict__ invstd, RowOrder order, int nchunks,
+                                               unsigned tiles, int HW, unsigned P) {
     const unsigned tile = blockIdx.x % tiles;
     const int ck = static_cast<int>(blockIdx.x / tiles);
     const unsigned p = (tile * kThreads + threadIdx.x) * V;
     const typename T::storage* xp = x + p;
+    const typename T::storage* rp = ACT && res ? res + p : nullptr;
     typename T::storage* yp = y + p;
-    // x is an input of the whole call, so the first rows can be requested before the statistics
-    // kernels ahead of this one have finished; only mean / invstd have to wait for them.
+    // x (and the residual) are inputs of the whole call, so the first rows can be requested before the
+    // statistics kernels ahead of this one have finished; only mean / invstd have to wait for them.
     // Rows go in batches of kUnroll with all loads of a batch in flight together; the last batch may be short.
     int i = ck;
-    Vec<T, V> v[kUnroll];
+    Vec<T, V> v[kUnroll], vr[kUnroll];
     int row[kUnroll];
     if (p < P) {
 #pragma unroll
@@ -707,6 +712,7 @@ col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::stor
             if (i + u * nchunks < order.rows) {
                 row[u] = order(i + u * nchunks);
                 v[u].load(xp + static_cast<size_t>(row[u]) * P);
+                if (ACT && rp) vr[u].load(rp + static_cast<size_t>(row[u]) * P);
             }
         }
     }
@@ -728,7 +734,14 @@ col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::stor
         for (int u = 0; u < kUnroll; ++u) {
             if (i + u * nchunks < order.rows) {
 #pragma unroll
-                for (int j = 0; j < V; ++j) v[u].set(j, fmaf(a[j], v[u].get(j), b[j]));
+                for (int j = 0; j < V; ++j) {
+                    float z = fmaf(a[j], v[u].get(j), b[j]);
+                    if (ACT) {
+                        if (rp) z += vr[u].get(j);
+                        z = fmaxf(z, 0.f);
+                    }
+                    v[u].set(j, z);
+                }
                 v[u].store(yp + static_cast<size_t>(row[u]) * P);
             }
         }
@@ -739,9 +752,18 @@ col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::stor
             if (i + u * nchunks < order.rows) {
                 row[u] = order(i + u * nchunks);
                 v[u].load(xp + static_cast<size_t>(row[u]) * P);
+                if (ACT && rp) vr[u].load(rp + static_cast<size_t>(row[u]) * P);
             }
         }
     }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+col_normalize_kernel(const typename T::storage* __restrict__ x, typename T::storage* __restrict__ y,
+                     const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
+                     const float* __restrict__ invstd, RowOrder order, int nchunks, unsigned tiles, int HW, unsigned P) {
+    normalize_rows<T, V, false>(x, nullptr, y, gamma, beta, mean, invstd, order, nchunks, tiles, HW, P);
 }
 
 // ------------------------------------------------------------------------------------ backward, pass 1
@@ -788,12 +810,20 @@ __device__ __forceinline__ void fold_thread_sums(const float2* s_first, const fl
 // (few registers, four blocks per SM even for bf16; pays extra arithmetic in every warp that holds a
 // thread straddling two maps - right for large maps, where such threads are rare) or per position (no
 // special case for straddling threads - right for small maps, where most warps hold one).
-template <typename T, int V, bool WRITE_DX, bool PER_CHANNEL>
-__global__ void __launch_bounds__(kThreads, PER_CHANNEL ? 4 : 3)
-col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
-                      typename T::storage* __restrict__ dx, const float* __restrict__ gamma,
-                      const float* __restrict__ mean, const float* __restrict__ invstd, RowOrder order, int nchunks,
-                      unsigned tiles, int HW, unsigned P, bool virtual_pass, GradSink G) {
+// With ACT (per-position sums only) the layer is followed by the fused residual add + ReLU: the gradient that
+// enters every formula is g = dy where a x + b + r > 0, else 0 (the mask is recomputed from x and r instead
+// of being stored), and dr = g is written to `dres` when given.
+template <typename T, int V, bool WRITE_DX, bool PER_CHANNEL, bool ACT>
+__device__ __forceinline__ void bwd_reduce_rows(const typename T::storage* __restrict__ x,
+                                                const typename T::storage* __restrict__ res,
+                                                const typename T::storage* __restrict__ dy,
+                                                typename T::storage* __restrict__ dx,
+                                                typename T::storage* __restrict__ dres,
+                                                const float* __restrict__ gamma, const float* __restrict__ beta,
+                                                const float* __restrict__ mean, const float* __restrict__ invstd,
+                                                RowOrder order, int nchunks, unsigned tiles, int HW, unsigned P,
+                                                bool virtual_pass, GradSink G) {
+    static_assert(!ACT || (WRITE_DX && !PER_CHANNEL), "the fused activation uses the per-position sums");
     constexpr unsigned TP = kThreads * V;
     // per-position sums (maps smaller than a vector) or, reusing the space, per-thread sums
     __shared__ __align__(16) float s_sums[2 * TP];
@@ -896,16 +926,19 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
 #pragma unroll
         for (int j = 0; j < V; ++j) acc_dy[j] = acc_dyxc[j] = 0.f;
         if (p < P) {
-            float a[V], mu[V];
+            float a[V], mu[V], b[V];
             if (HW >= V) {  // at most two channels per thread: two parameter sets, selected per position
                 const TwoChannels ch(p, HW, V);
                 const float mu0 = mean[ch.c0], mu1 = mean[ch.c1];
                 const float a0 = WRITE_DX ? gamma[ch.c0] * invstd[ch.c0] : 0.f;
                 const float a1 = WRITE_DX ? gamma[ch.c1] * invstd[ch.c1] : 0.f;
+                const float b0 = ACT ? fmaf(-mu0, a0, beta[ch.c0]) : 0.f;
+                const float b1 = ACT ? fmaf(-mu1, a1, beta[ch.c1]) : 0.f;
 #pragma unroll
                 for (int j = 0; j < V; ++j) {
                     mu[j] = ch.pick(j, mu0, mu1);
                     a[j] = ch.pick(j, a0, a1);
+                    b[j] = ch.pick(j, b0, b1);
                 }
             } else {
                 int c[V];
@@ -914,10 +947,13 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
                 for (int j = 0; j < V; ++j) {
                     mu[j] = mean[c[j]];
                     a[j] = WRITE_DX ? gamma[c[j]] * invstd[c[j]] : 0.f;
+                    b[j] = ACT ? fmaf(-mu[j], a[j], beta[c[j]]) : 0.f;
                 }
             }
+            const typename T::storage* rp = ACT && res ? res + p : nullptr;
+            typename T::storage* drp = ACT && dres ? dres + p : nullptr;
             for (int i = ck; i < order.rows; i += kUnroll * nchunks) {
-                Vec<T, V> vx[kUnroll], vg[kUnroll];
+                Vec<T, V> vx[kUnroll], vg[kUnroll], vr[kUnroll];
                 int row[kUnroll];
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
@@ -925,6 +961,7 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
                         row[u] = order(i + u * nchunks);
                         vx[u].load(xp + static_cast<size_t>(row[u]) * P);
                         vg[u].load(gp + static_cast<size_t>(row[u]) * P);
+                        if (ACT && rp) vr[u].load(rp + static_cast<size_t>(row[u]) * P);
                     }
                 }
 #pragma unroll
@@ -933,6 +970,17 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
                         float g[V], xv[V];
                         vg[u].unpack(g);
                         vx[u].unpack(xv);
+                        if (ACT) {
+                            float r[V];
+                            if (rp) vr[u].unpack(r);
+#pragma unroll
+                            for (int j = 0; j < V; ++j)
+                                g[j] = fmaf(a[j], xv[j], b[j]) + (rp ? r[j] : 0.f) > 0.f ? g[j] : 0.f;
+                            if (drp) {
+                                vr[u].pack(g);
+                                vr[u].store(drp + static_cast<size_t>(row[u]) * P);
+                            }
+                        }
 #pragma unroll
                         for (int j = 0; j < V; ++j) {
                             acc_dy[j] += g[j];
@@ -957,6 +1005,16 @@ col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
     }
 }
 
+template <typename T, int V, bool WRITE_DX, bool PER_CHANNEL>
+__global__ void __launch_bounds__(kThreads, PER_CHANNEL ? 4 : 3)
+col_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
+                      typename T::storage* __restrict__ dx, const float* __restrict__ gamma,
+                      const float* __restrict__ mean, const float* __restrict__ invstd, RowOrder order, int nchunks,
+                      unsigned tiles, int HW, unsigned P, bool virtual_pass, GradSink G) {
+    bwd_reduce_rows<T, V, WRITE_DX, PER_CHANNEL, false>(x, nullptr, dy, dx, nullptr, gamma, nullptr, mean, invstd, order,
+                                                        nchunks, tiles, HW, P, virtual_pass, G);
+}
+
 // ------------------------------------------------------------------------------------ backward, statistics terms
 // Per-channel coefficients of the full gradient of a sampled element (upper branch of Eq. 6):
 //   dx = a dy - A - Q (x - mean),  a = gamma invstd,  A = a dbeta / s,  Q = a invstd dgamma / s.
@@ -974,16 +1032,27 @@ __device__ __forceinline__ FixCoef fix_coef(float gamma, float mean, float invst
     return k;
 }
 
+// masked gradient of one element under the fused residual add + ReLU: dy where the pre-activation is positive
+__device__ __forceinline__ float act_gradient(float a, float b, float x, float r, float dy) {
+    return fmaf(a, x, b) + r > 0.f ? dy : 0.f;
+}
+
 // Rows given by `list` (or begin .. begin+count-1): dx = a dy - A - Q (x - mean); dy == NULL reads as zeros.
 // With `fold` the kernel finishes the sums of Eq. 5 itself from the partials in G (see block_finish_grads)
-// and dgamma / dbeta are not read.
-template <typename T, int V>
-__global__ void __launch_bounds__(kThreads)
-col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
-                 typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
-                 const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
-                 float inv_s, const int* __restrict__ list, int begin, RowOrder order, int nchunks, unsigned tiles,
-                 int HW, unsigned P, GradSink G, int fold) {
+// and dgamma / dbeta are not read.  With ACT the masked gradient takes the place of dy (see bwd_reduce_rows).
+template <typename T, int V, bool ACT>
+__device__ __forceinline__ void fixup_rows(const typename T::storage* __restrict__ x,
+                                           const typename T::storage* __restrict__ res,
+                                           const typename T::storage* __restrict__ dy,
+                                           typename T::storage* __restrict__ dx, const float* __restrict__ gamma,
+                                           const float* __restrict__ beta, const float* __restrict__ mean,
+                                           const float* __restrict__ invstd, const float* __restrict__ dgamma,
+                                           const float* __restrict__ dbeta, float inv_s, const int* __restrict__ list,
+                                           int begin, RowOrder order, int nchunks, unsigned tiles, int HW, unsigned P,
+                                           GradSink G, int fold) {
+    // rows in flight per thread: the fused activation reads a third tensor, and its pass over a whole tensor
+    // (full BN) measured faster with fewer registers and more resident blocks than with deeper batches
+    constexpr int U = ACT ? 2 : kUnroll;
     __shared__ float2 s_grad[kFoldSlots];
     grid_dependency_wait();
     grid_dependency_launch();
@@ -994,6 +1063,7 @@ col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::st
     if (fold) block_finish_grads(G, tc.c_first, tc.nslots, HW, ck == 0, tile, kThreads * V, HW, s_grad);
     if (p >= P) return;
     FixCoef k[V];
+    float b[V];
     {
         int c[V];
         position_channels<V>(p, HW, c);
@@ -1001,25 +1071,30 @@ col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::st
         for (int j = 0; j < V; ++j) {
             const float2 g = fold ? s_grad[c[j] - tc.c_first] : make_float2(dgamma[c[j]], dbeta[c[j]]);
             k[j] = fix_coef(gamma[c[j]], mean[c[j]], invstd[c[j]], g.x, g.y, inv_s);
+            b[j] = ACT ? fmaf(-k[j].mu, k[j].a, beta[c[j]]) : 0.f;
         }
     }
+    const bool with_res = ACT && res;
     int i = ck;
-    for (; i + (kUnroll - 1) * nchunks < order.rows; i += kUnroll * nchunks) {
-        Vec<T, V> vx[kUnroll], vg[kUnroll];
-        int row[kUnroll];
+    for (; i + (U - 1) * nchunks < order.rows; i += U * nchunks) {
+        Vec<T, V> vx[U], vg[U], vr[U];
+        int row[U];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < U; ++u) {
             int v = order(i + u * nchunks);
             row[u] = list ? list[v] : begin + v;
             vx[u].load(x + static_cast<size_t>(row[u]) * P + p);
             if (dy) vg[u].load(dy + static_cast<size_t>(row[u]) * P + p);
+            if (with_res) vr[u].load(res + static_cast<size_t>(row[u]) * P + p);
         }
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < U; ++u) {
 #pragma unroll
             for (int j = 0; j < V; ++j) {
                 float g = dy ? vg[u].get(j) : 0.f;
-                vg[u].set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (vx[u].get(j) - k[j].mu));
+                const float xv = vx[u].get(j);
+                if (ACT) g = act_gradient(k[j].a, b[j], xv, with_res ? vr[u].get(j) : 0.f, g);
+                vg[u].set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (xv - k[j].mu));
             }
             vg[u].store(dx + static_cast<size_t>(row[u]) * P + p);
         }
@@ -1028,26 +1103,43 @@ col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::st
         int v = order(i);
         int n = list ? list[v] : begin + v;
         size_t off = static_cast<size_t>(n) * P + p;
-        Vec<T, V> vx, vg;
+        Vec<T, V> vx, vg, vr;
         vx.load(x + off);
         if (dy) vg.load(dy + off);
+        if (with_res) vr.load(res + off);
 #pragma unroll
         for (int j = 0; j < V; ++j) {
             float g = dy ? vg.get(j) : 0.f;
-            vg.set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (vx.get(j) - k[j].mu));
+            const float xv = vx.get(j);
+            if (ACT) g = act_gradient(k[j].a, b[j], xv, with_res ? vr.get(j) : 0.f, g);
+            vg.set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (xv - k[j].mu));
         }
         vg.store(dx + off);
     }
 }
 
-// The same for the patch elements (compact positions, see PatchThread).
-template <typename T>
+template <typename T, int V>
 __global__ void __launch_bounds__(kThreads)
-patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
-                   typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
-                   const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
-                   float inv_s, PatchRule rule, int N, int C, int H, int W, int nchunks, unsigned tiles,
-                   unsigned* status, GradSink G, int fold) {
+col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
+                 typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
+                 const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
+                 float inv_s, const int* __restrict__ list, int begin, RowOrder order, int nchunks, unsigned tiles,
+                 int HW, unsigned P, GradSink G, int fold) {
+    fixup_rows<T, V, false>(x, nullptr, dy, dx, gamma, nullptr, mean, invstd, dgamma, dbeta, inv_s, list, begin, order,
+                            nchunks, tiles, HW, P, G, fold);
+}
+
+// The same for the patch elements (compact positions, see PatchThread).
+template <typename T, bool ACT>
+__device__ __forceinline__ void patch_fixup_rows(const typename T::storage* __restrict__ x,
+                                                 const typename T::storage* __restrict__ res,
+                                                 const typename T::storage* __restrict__ dy,
+                                                 typename T::storage* __restrict__ dx, const float* __restrict__ gamma,
+                                                 const float* __restrict__ beta, const float* __restrict__ mean,
+                                                 const float* __restrict__ invstd, const float* __restrict__ dgamma,
+                                                 const float* __restrict__ dbeta, float inv_s, PatchRule rule, int N,
+                                                 int C, int H, int W, int nchunks, unsigned tiles, unsigned* status,
+                                                 GradSink G, int fold) {
     __shared__ float2 s_grad[kFoldSlots];
     grid_dependency_wait();
     grid_dependency_launch();
@@ -1062,24 +1154,42 @@ patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::
     const size_t P = static_cast<size_t>(C) * H * W;
     const float2 grads = fold ? s_grad[me.c - tc.c_first] : make_float2(dgamma[me.c], dbeta[me.c]);
     const FixCoef k = fix_coef(gamma[me.c], mean[me.c], invstd[me.c], grads.x, grads.y, inv_s);
+    const float b = ACT ? fmaf(-k.mu, k.a, beta[me.c]) : 0.f;
+    const bool with_res = ACT && res;
     int n = ck;
     for (; n + (kUnroll - 1) * nchunks < N; n += kUnroll * nchunks) {
         size_t at[kUnroll];
-        float g[kUnroll], xv[kUnroll];
+        float g[kUnroll], xv[kUnroll], r[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
             at[u] = me.at(rule, n + u * nchunks, P, H, W, status);
             g[u] = to_float<T>(dy[at[u]]);
             xv[u] = to_float<T>(x[at[u]]);
+            r[u] = with_res ? to_float<T>(res[at[u]]) : 0.f;
         }
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) dx[at[u]] = from_float<T>(fmaf(k.a, g[u], -k.A) - k.Q * (xv[u] - k.mu));
+        for (int u = 0; u < kUnroll; ++u) {
+            if (ACT) g[u] = act_gradient(k.a, b, xv[u], r[u], g[u]);
+            dx[at[u]] = from_float<T>(fmaf(k.a, g[u], -k.A) - k.Q * (xv[u] - k.mu));
+        }
     }
     for (; n < N; n += nchunks) {
         size_t at = me.at(rule, n, P, H, W, status);
         float g = to_float<T>(dy[at]), xv = to_float<T>(x[at]);
+        if (ACT) g = act_gradient(k.a, b, xv, with_res ? to_float<T>(res[at]) : 0.f, g);
         dx[at] = from_float<T>(fmaf(k.a, g, -k.A) - k.Q * (xv - k.mu));
     }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
+                   typename T::storage* __restrict__ dx, const float* __restrict__ gamma, const float* __restrict__ mean,
+                   const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
+                   float inv_s, PatchRule rule, int N, int C, int H, int W, int nchunks, unsigned tiles,
+                   unsigned* status, GradSink G, int fold) {
+    patch_fixup_rows<T, false>(x, nullptr, dy, dx, gamma, nullptr, mean, invstd, dgamma, dbeta, inv_s, rule, N, C, H, W,
+                               nchunks, tiles, status, G, fold);
 }
 
 // ------------------------------------------------------------------------------------ small sampled sets: one block per channel
@@ -1341,69 +1451,15 @@ per_point_shares_kernel(const float* __restrict__ sums, const float* __restrict_
 // The step that follows a BN layer in a residual network, fused so that the pre-activation tensor is
 // never written: forward y = max(0, a x + b + r); backward g = dy where a x + b + r > 0, else 0, and g
 // takes the place of dy everywhere (sums, dx, statistics terms); dr = g.  The mask is recomputed from
-// x (and r) instead of being stored.  r / dr may be NULL.  These kernels mirror col_normalize,
-// col_bwd_reduce, col_fixup and patch_fixup; they are kept apart from them on purpose.
-struct ActCoef {
-    float a, b;  // z = a x + b (+ r)
-};
-
+// x (and r) instead of being stored.  r / dr may be NULL.  These are the ACT instances of the bodies of
+// col_normalize, col_bwd_reduce, col_fixup and patch_fixup.
 template <typename T, int V>
 __global__ void __launch_bounds__(kThreads)
 act_normalize_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ res,
                      typename T::storage* __restrict__ y, const float* __restrict__ gamma,
                      const float* __restrict__ beta, const float* __restrict__ mean, const float* __restrict__ invstd,
-                     int rows, int nchunks, unsigned tiles, int HW, unsigned P) {
-    const unsigned tile = blockIdx.x % tiles;
-    const int ck = static_cast<int>(blockIdx.x / tiles);
-    const unsigned p = (tile * kThreads + threadIdx.x) * V;
-    // x and the residual are inputs of the whole call: the first batch of rows is requested before the
-    // statistics kernels ahead of this one have finished (as in col_normalize_kernel)
-    int i = ck;
-    Vec<T, V> vx[kUnroll], vr[kUnroll];
-    if (p < P) {
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
-            if (i + u * nchunks < rows) {
-                const size_t off = static_cast<size_t>(i + u * nchunks) * P + p;
-                vx[u].load(x + off);
-                if (res) vr[u].load(res + off);
-            }
-    }
-    grid_dependency_wait();
-    grid_dependency_launch();
-    if (p >= P) return;
-    float a[V], b[V];
-    {
-        int c[V];
-        position_channels<V>(p, HW, c);
-#pragma unroll
-        for (int j = 0; j < V; ++j) {
-            a[j] = gamma[c[j]] * invstd[c[j]];
-            b[j] = fmaf(-mean[c[j]], a[j], beta[c[j]]);
-        }
-    }
-    while (true) {
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
-            if (i + u * nchunks < rows) {
-#pragma unroll
-                for (int j = 0; j < V; ++j) {
-                    float z = fmaf(a[j], vx[u].get(j), b[j]);
-                    if (res) z += vr[u].get(j);
-                    vx[u].set(j, fmaxf(z, 0.f));
-                }
-                vx[u].store(y + static_cast<size_t>(i + u * nchunks) * P + p);
-            }
-        i += kUnroll * nchunks;
-        if (i >= rows) break;
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
-            if (i + u * nchunks < rows) {
-                const size_t off = static_cast<size_t>(i + u * nchunks) * P + p;
-                vx[u].load(x + off);
-                if (res) vr[u].load(res + off);
-            }
-    }
+                     RowOrder order, int nchunks, unsigned tiles, int HW, unsigned P) {
+    normalize_rows<T, V, true>(x, res, y, gamma, beta, mean, invstd, order, nchunks, tiles, HW, P);
 }
 
 template <typename T, int V>
@@ -1412,74 +1468,9 @@ act_bwd_reduce_kernel(const typename T::storage* __restrict__ x, const typename 
                       const typename T::storage* __restrict__ dy, typename T::storage* __restrict__ dx,
                       typename T::storage* __restrict__ dres, const float* __restrict__ gamma,
                       const float* __restrict__ beta, const float* __restrict__ mean, const float* __restrict__ invstd,
-                      int rows, int nchunks, unsigned tiles, int HW, unsigned P, GradSink G) {
-    constexpr unsigned TP = kThreads * V;
-    __shared__ float s_dy[TP];
-    __shared__ float s_dyxc[TP];
-    grid_dependency_wait();
-    grid_dependency_launch();
-    const unsigned tile = blockIdx.x % tiles;
-    const int ck = static_cast<int>(blockIdx.x / tiles);
-    const unsigned p = (tile * kThreads + threadIdx.x) * V;
-    float acc_dy[V], acc_dyxc[V];
-#pragma unroll
-    for (int j = 0; j < V; ++j) acc_dy[j] = acc_dyxc[j] = 0.f;
-    if (p < P) {
-        float a[V], b[V], mu[V];
-        {
-            int c[V];
-            position_channels<V>(p, HW, c);
-#pragma unroll
-            for (int j = 0; j < V; ++j) {
-                mu[j] = mean[c[j]];
-                a[j] = gamma[c[j]] * invstd[c[j]];
-                b[j] = fmaf(-mu[j], a[j], beta[c[j]]);
-            }
-        }
-        // batches of kUnroll rows, all loads of a batch in flight together; the last batch may be short
-        for (int i = ck; i < rows; i += kUnroll * nchunks) {
-            Vec<T, V> vx[kUnroll], vg[kUnroll], vr[kUnroll];
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u)
-                if (i + u * nchunks < rows) {
-                    const size_t off = static_cast<size_t>(i + u * nchunks) * P + p;
-                    vx[u].load(x + off);
-                    vg[u].load(dy + off);
-                    if (res) vr[u].load(res + off);
-                }
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u)
-                if (i + u * nchunks < rows) {
-                    const size_t off = static_cast<size_t>(i + u * nchunks) * P + p;
-#pragma unroll
-                    for (int j = 0; j < V; ++j) {
-                        const float xv = vx[u].get(j);
-                        float z = fmaf(a[j], xv, b[j]);
-                        if (res) z += vr[u].get(j);
-                        const float g = z > 0.f ? vg[u].get(j) : 0.f;
-                        acc_dy[j] += g;
-                        acc_dyxc[j] = fmaf(g, xv - mu[j], acc_dyxc[j]);
-                        vg[u].set(j, g);
-                        vx[u].set(j, a[j] * g);
-                    }
-                    vx[u].store(dx + off);
-                    if (dres) vg[u].store(dres + off);
-                }
-        }
-    }
-#pragma unroll
-    for (int j = 0; j < V; ++j) {
-        s_dy[threadIdx.x * V + j] = acc_dy[j];
-        s_dyxc[threadIdx.x * V + j] = acc_dyxc[j];
-    }
-    __syncthreads();
-    fold_sums(s_dy, s_dyxc, TileChannels(tile, TP, P, HW), HW,
-              G.partials + (static_cast<size_t>(ck) * tiles + tile) * G.L.max_slots);
-}
-
-// masked gradient of one element: dy where the pre-activation is positive
-__device__ __forceinline__ float act_gradient(float a, float b, float x, float r, float dy) {
-    return fmaf(a, x, b) + r > 0.f ? dy : 0.f;
+                      RowOrder order, int nchunks, unsigned tiles, int HW, unsigned P, GradSink G) {
+    bwd_reduce_rows<T, V, true, false, true>(x, res, dy, dx, dres, gamma, beta, mean, invstd, order, nchunks, tiles, HW,
+                                             P, false, G);
 }
 
 template <typename T, int V>
@@ -1488,40 +1479,10 @@ act_col_fixup_kernel(const typename T::storage* __restrict__ x, const typename T
                      const typename T::storage* __restrict__ dy, typename T::storage* __restrict__ dx,
                      const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
                      const float* __restrict__ invstd, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
-                     float inv_s, const int* __restrict__ list, int begin, int count, int nchunks, unsigned tiles,
-                     int HW, unsigned P) {
-    grid_dependency_wait();
-    grid_dependency_launch();
-    const unsigned tile = blockIdx.x % tiles;
-    const int ck = static_cast<int>(blockIdx.x / tiles);
-    const unsigned p = (tile * kThreads + threadIdx.x) * V;
-    if (p >= P) return;
-    FixCoef k[V];
-    float b[V];
-    {
-        int c[V];
-        position_channels<V>(p, HW, c);
-#pragma unroll
-        for (int j = 0; j < V; ++j) {
-            k[j] = fix_coef(gamma[c[j]], mean[c[j]], invstd[c[j]], dgamma[c[j]], dbeta[c[j]], inv_s);
-            b[j] = fmaf(-k[j].mu, k[j].a, beta[c[j]]);
-        }
-    }
-    for (int i = ck; i < count; i += nchunks) {
-        const int n = list ? list[i] : begin + i;
-        const size_t off = static_cast<size_t>(n) * P + p;
-        Vec<T, V> vx, vg, vr;
-        vx.load(x + off);
-        vg.load(dy + off);
-        if (res) vr.load(res + off);
-#pragma unroll
-        for (int j = 0; j < V; ++j) {
-            const float xv = vx.get(j);
-            const float g = act_gradient(k[j].a, b[j], xv, res ? vr.get(j) : 0.f, vg.get(j));
-            vg.set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (xv - k[j].mu));
-        }
-        vg.store(dx + off);
-    }
+                     float inv_s, const int* __restrict__ list, int begin, RowOrder order, int nchunks, unsigned tiles,
+                     int HW, unsigned P, GradSink G, int fold) {
+    fixup_rows<T, V, true>(x, res, dy, dx, gamma, beta, mean, invstd, dgamma, dbeta, inv_s, list, begin, order, nchunks,
+                           tiles, HW, P, G, fold);
 }
 
 template <typename T>
@@ -1531,23 +1492,9 @@ act_patch_fixup_kernel(const typename T::storage* __restrict__ x, const typename
                        const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ mean,
                        const float* __restrict__ invstd, const float* __restrict__ dgamma,
                        const float* __restrict__ dbeta, float inv_s, PatchRule rule, int N, int C, int H, int W,
-                       int nchunks, unsigned tiles, unsigned* status) {
-    grid_dependency_wait();
-    grid_dependency_launch();
-    const unsigned tile = blockIdx.x % tiles;
-    const int ck = static_cast<int>(blockIdx.x / tiles);
-    const unsigned j = tile * kThreads + threadIdx.x;
-    if (j >= static_cast<unsigned>(C) * rule.ph * rule.pw) return;
-    const PatchThread me(j, rule, H, W);
-    const size_t P = static_cast<size_t>(C) * H * W;
-    const FixCoef k = fix_coef(gamma[me.c], mean[me.c], invstd[me.c], dgamma[me.c], dbeta[me.c], inv_s);
-    const float b = fmaf(-k.mu, k.a, beta[me.c]);
-    for (int n = ck; n < N; n += nchunks) {
-        const size_t at = me.at(rule, n, P, H, W, status);
-        const float xv = to_float<T>(x[at]);
-        const float g = act_gradient(k.a, b, xv, res ? to_float<T>(res[at]) : 0.f, to_float<T>(dy[at]));
-        dx[at] = from_float<T>(fmaf(k.a, g, -k.A) - k.Q * (xv - k.mu));
-    }
+                       int nchunks, unsigned tiles, unsigned* status, GradSink G, int fold) {
+    patch_fixup_rows<T, true>(x, res, dy, dx, gamma, beta, mean, invstd, dgamma, dbeta, inv_s, rule, N, C, H, W, nchunks,
+                              tiles, status, G, fold);
 }
 
 // ------------------------------------------------------------------------------------ selection mask (test aid)
