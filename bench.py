@@ -545,7 +545,7 @@ def measure_workload(torch, dist, bns, args, layers, inputs, local, world, secon
     return res, dev
 
 
-OTHER_CONFIGS = ["cifar", "vdn", "resnet50", "fs_vdn", "fs_relu"]
+OTHER_CONFIGS = ["tiny", "cifar", "vdn", "resnet50", "fs_vdn", "fs_relu"]
 
 
 def run_ours(args):
@@ -633,7 +633,7 @@ def run_ours(args):
             olayers = workload_layers(name)
             oin = [device_inputs(l, layer_seed(name, i), torch) for i, l in enumerate(olayers)]
             res, odev = measure_workload(torch, dist, bns, oargs, olayers, oin, local, world, args.seconds / 2,
-                                         args.seconds / 8, warm=name in ("cifar", "vdn"))
+                                         args.seconds / 8, warm=name in ("tiny", "cifar", "vdn"))
             res["steps_per_repeat"] = oargs.steps
             res["frac_of_hbm_peak"] = round(res["value"] / peak, 4)
             res["frac_of_nominal_8TBps"] = round(res["value"] / NOMINAL_HBM_GBS, 4)
