@@ -259,6 +259,178 @@ nhwc_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::s
     }
 }
 
+// ------------------------------------------------------------------------------------ small sampled sets
+// When the sampled set is a few thousand rows (small patches, a couple of samples) one block per narrow
+// strip of channels can visit all of it: the statistics then need no partials and no finalize launch, and
+// in the backward the block that combines the strip's partial sums applies the statistics terms to the
+// strip's sampled elements right away.  The grid is (1, strips); a block is CW (1 or 2) channel-vectors
+// wide - 32 bytes of every sampled row - and kThreads / CW row-lanes deep.
+constexpr int kNhwcDirectUnroll = 8;  // rows a thread keeps in flight
+
+// Sum over the row-lanes of a block, in a fixed order: lanes of a warp by a shuffle tree (a warp holds
+// 32 / CW row-lanes of each channel-vector, CW a power of two), then the warps through shared memory.
+// The totals land in shared memory: s_out[cvi * NV + i] for value i of channel-vector cvi of the block.
+template <int NV>
+__device__ __forceinline__ void nhwc_block_sum(float (&val)[NV], int CW, float* s_warp, float* s_out) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+    for (int i = 0; i < NV; ++i)
+        for (int d = CW; d < 32; d <<= 1) val[i] += __shfl_xor_sync(0xffffffffu, val[i], d);
+    if (lane < CW) {
+#pragma unroll
+        for (int i = 0; i < NV; ++i) s_warp[(warp * 2 + lane) * NV + i] = val[i];
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < CW * NV; e += kThreads) {
+        const int cvi = e / NV, i = e - cvi * NV;
+        float tot = 0.f;
+        for (int w = 0; w < kThreads / 32; ++w) tot += s_warp[(w * 2 + cvi) * NV + i];
+        s_out[e] = tot;
+    }
+    __syncthreads();
+}
+
+// mean and invstd of the block's channels straight from the sampled rows.  Sums are shifted by the value of
+// the first sampled row (one pivot per channel for the whole block, so the lanes' sums simply add).
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+nhwc_direct_moments_kernel(const typename T::storage* __restrict__ x, RowSet set, NhwcShape s, float eps,
+                           float* __restrict__ mean, float* __restrict__ invstd, unsigned* status) {
+    constexpr int U = kNhwcDirectUnroll;
+    __shared__ float s_warp[(kThreads / 32) * 2 * 2 * V];
+    __shared__ float s_tot[2 * 2 * V];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const NhwcThread me(s);
+    float K[V], sums[2 * V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) K[j] = sums[j] = sums[V + j] = 0.f;
+    if (me.active) {
+        const typename T::storage* xp = x + static_cast<size_t>(me.cv) * V;
+        Vec<T, V> first;
+        first.load(xp + static_cast<size_t>(set.row(0, status)) * s.C);
+#pragma unroll
+        for (int j = 0; j < V; ++j) K[j] = first.get(j);
+        for (int q = me.rl; q < set.total; q += U * s.RL) {
+            Vec<T, V> v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (q + u * s.RL < set.total) v[u].load(xp + static_cast<size_t>(set.row(q + u * s.RL, status)) * s.C);
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (q + u * s.RL < set.total) {
+#pragma unroll
+                    for (int j = 0; j < V; ++j) {
+                        const float d = v[u].get(j) - K[j];
+                        sums[j] += d;
+                        sums[V + j] = fmaf(d, d, sums[V + j]);
+                    }
+                }
+        }
+    }
+    nhwc_block_sum<2 * V>(sums, s.CW, s_warp, s_tot);
+    // thread (rl == 0, cvi) finishes the V channels of its vector; it holds their pivots
+    if (me.active && me.rl == 0) {
+        const int cvi = threadIdx.x % s.CW;
+        const float n = static_cast<float>(set.total);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            const float s1 = s_tot[cvi * 2 * V + j], s2 = s_tot[cvi * 2 * V + V + j];
+            const float m2 = fmaxf(s2 - s1 * s1 / n, 0.f);
+            mean[me.cv * V + j] = K[j] + s1 / n;
+            invstd[me.cv * V + j] = 1.0f / sqrtf(m2 / n + eps);
+        }
+    }
+}
+
+// Backward for a small sampled set: the block adds up the partial sums that pass 1 left for its channels
+// (every block of pass 1 wrote one per channel), publishes dgamma / dbeta, and rewrites the gradient of the
+// strip's sampled elements with the statistics terms.  dy == NULL reads as zeros; dx == NULL skips the rewrite.
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+nhwc_direct_finalize_fixup_kernel(const typename T::storage* __restrict__ x, const typename T::storage* __restrict__ dy,
+                                  typename T::storage* __restrict__ dx, const float* __restrict__ gamma,
+                                  const float* __restrict__ mean, const float* __restrict__ invstd,
+                                  const float2* __restrict__ partials, int entries,
+                                  const float2* __restrict__ partials_v, int entries_v, float inv_s, RowSet set,
+                                  NhwcShape s, float* __restrict__ dgamma, float* __restrict__ dbeta, unsigned* status) {
+    constexpr int U = kNhwcDirectUnroll;
+    __shared__ float2 s_part[kThreads];
+    __shared__ float2 s_grad[2 * V];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    const NhwcThread me(s);
+    // partial sums: thread t adds the entries el, el + lanes, ... of channel ch of the strip (neighbouring threads
+    // read neighbouring channels of one entry), then thread ch adds the lanes' results in lane order
+    const int nch = s.CW * V, lanes = kThreads / nch;
+    const int ch = threadIdx.x % nch, el = threadIdx.x / nch;
+    const int c_of_ch = blockIdx.y * nch + ch;
+    float sa = 0.f, sb = 0.f;
+    if (el < lanes && c_of_ch < s.C) {
+        for (int pass = 0; pass < 2; ++pass) {
+            const float2* src = pass ? partials_v : partials;
+            const int n = pass ? entries_v : entries;
+            if (!src) continue;
+            for (int e = el; e < n; e += U * lanes) {  // batches of U loads in flight, added in entry order
+                float2 v[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    v[u] = e + u * lanes < n ? src[static_cast<size_t>(e + u * lanes) * s.C + c_of_ch] : make_float2(0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    sa += v[u].x;
+                    sb += v[u].y;
+                }
+            }
+        }
+    }
+    s_part[threadIdx.x] = make_float2(sa, sb);
+    __syncthreads();
+    if (threadIdx.x < nch && c_of_ch < s.C) {
+        float ta = 0.f, tb = 0.f;
+        for (int l = 0; l < lanes; ++l) {
+            ta += s_part[l * nch + threadIdx.x].x;
+            tb += s_part[l * nch + threadIdx.x].y;
+        }
+        tb *= invstd[c_of_ch];
+        dbeta[c_of_ch] = ta;
+        dgamma[c_of_ch] = tb;
+        s_grad[threadIdx.x] = make_float2(tb, ta);  // (dgamma, dbeta)
+    }
+    __syncthreads();
+    if (!dx || !me.active) return;
+    FixCoef k[V];
+    const int cvi = threadIdx.x % s.CW;
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        const int c = me.cv * V + j;
+        const float2 g = s_grad[cvi * V + j];
+        k[j] = fix_coef(gamma[c], mean[c], invstd[c], g.x, g.y, inv_s);
+    }
+    const size_t col = static_cast<size_t>(me.cv) * V;
+    for (int q = me.rl; q < set.total; q += U * s.RL) {
+        Vec<T, V> vx[U], vg[U];
+        size_t off[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (q + u * s.RL < set.total) {
+                off[u] = static_cast<size_t>(set.row(q + u * s.RL, status)) * s.C + col;
+                vx[u].load(x + off[u]);
+                if (dy) vg[u].load(dy + off[u]);
+            }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (q + u * s.RL < set.total) {
+#pragma unroll
+                for (int j = 0; j < V; ++j) {
+                    const float g = dy ? vg[u].get(j) : 0.f;
+                    vg[u].set(j, fmaf(k[j].a, g, -k[j].A) - k[j].Q * (vx[u].get(j) - k[j].mu));
+                }
+                vg[u].store(dx + off[u]);
+            }
+    }
+}
+
 // ------------------------------------------------------------------------------------ combining the blocks' partials
 // Every block of a channels-last pass leaves one partial per channel: partial[block*C + c].  Here lane l
 // of a warp owns channel 32*blockIdx.x + l (neighbouring lanes read neighbouring addresses) and the 32

@@ -360,9 +360,17 @@ NHWC_CASES = [
 @pytest.mark.parametrize("rule,kw", NHWC_CASES)
 @pytest.mark.parametrize("dtype,dims", [("f32", (12, 64, 9, 11)), ("bf16", (10, 40, 7, 7)), ("f32", (6, 7, 5, 3)),
                                         ("bf16", (3, 2080, 2, 2)), ("f32", (40, 16, 16, 16))])
-def test_channels_last_layout(rule, kw, dtype, dims):
-    """The NHWC entry points against the (NCHW) oracle on the transposed tensors."""
-    _check_channels_last(rule, kw, dtype, dims)
+@pytest.mark.parametrize("direct_max", [0, 8192])
+def test_channels_last_layout(rule, kw, dtype, dims, direct_max):
+    """The NHWC entry points against the (NCHW) oracle on the transposed tensors; once with small sampled sets
+    going through the one-block-per-strip kernels (the default) and once with every set going through partial
+    sums and the finalize launches."""
+    from paper_1810_10962_b200 import bns
+    try:
+        bns.set_tuning("direct_max", direct_max)
+        _check_channels_last(rule, kw, dtype, dims)
+    finally:
+        bns.set_tuning("direct_max", 8192)
 
 
 @pytest.mark.parametrize("rule,kw,dtype,dims", [
