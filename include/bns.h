@@ -388,7 +388,8 @@ const char* bns_kernel_name(int kernel_kind);
  * 32 MiB and more; "stat_target_blocks" / "stat_min_chunk": the same for the
  * statistics kernels; "direct_max": sampled elements per channel up to which one block per channel computes the
  * statistics (and, in the backward, combines the sums and applies the statistics terms) without
- * partial sums, 0 = never; "nhwc_blocks": blocks per launch of the channels-last kernels (each block leaves one partial per
+ * partial sums, 0 = never (the channels-last entry points have the same kind of path, one block per narrow strip
+ * of channels, for sampled sets of up to min(direct_max, 2048) pixel rows); "nhwc_blocks": blocks per launch of the channels-last kernels (each block leaves one partial per
  * channel); "slab": 0/1 use the one-launch path where it applies, "slab_cta_kb": preferred shared memory per block of
  * that path in KiB, "slab_min_ctas": grow its clusters while a launch has fewer blocks (0 = two per SM), "slab_max_mb":
  * tensors above this many MiB keep the streaming path (default 6: measured on B200, larger tensors run faster through
