@@ -972,7 +972,7 @@ struct NhwcLaunch {
 };
 
 // Block shape and grid for visiting `total` rows of C channels.
-NhwcLaunch plan_nhwc(int C, int ebytes, long total, bool statistics) {
+NhwcLaunch plan_nhwc(int C, int ebytes, long total, bool statistics, bool no_partials = false) {
     NhwcLaunch l{};
     int V = 16 / ebytes;
     while (V > 1 && C % V != 0) V >>= 1;
@@ -986,7 +986,12 @@ NhwcLaunch plan_nhwc(int C, int ebytes, long total, bool statistics) {
     // few, long-lived blocks: every block leaves one partial per channel, so the block count is also the
     // number of partials the finalize kernels have to read per channel
     (void)statistics;
-    const long target = std::max(1L, static_cast<long>(g_nhwc_blocks > 0 ? g_nhwc_blocks : sm_count() * 8) / gy);
+    // (a pass that leaves no partials - normalise - takes four times as many, shorter-lived blocks: measured 70 -> 64 us
+    // on 256x56x56x64 fp32.  Fewer blocks for the passes that do leave partials - four per SM - ran the ResNet-50 shapes
+    // 5 % faster, but then a thread adds up so many rows that the fp32 sums of the backward left the absolute
+    // tolerance on channels with a gradient near zero; compensated sums in double precision cost what was gained.)
+    const long blocks = static_cast<long>(g_nhwc_blocks > 0 ? g_nhwc_blocks : sm_count() * 8) * (no_partials ? 4 : 1);
+    const long target = std::max(1L, blocks / gy);
     long rpb = std::max<long>(static_cast<long>(s.RL) * kUnroll * 2, (total + target - 1) / target);
     rpb = (rpb + s.RL - 1) / s.RL * s.RL;
     s.rows_per_block = static_cast<int>(rpb);
@@ -1021,6 +1026,7 @@ struct NhwcProblem {
     long rows;                   // N*H*W
     long sampled_rows;           // rows in the sampled set (of x, or of xv for VIRTUAL)
     NhwcLaunch main, stat, virt; // all rows of x; the sampled rows; all rows of xv
+    NhwcLaunch norm, norm_virt;  // the same rows as main / virt for the normalise pass, which leaves no partials
     NhwcLaunch direct;           // the sampled rows, one block per strip of channels (small sets)
     bool small_set = false;      // few enough sampled rows for `direct`
     size_t off_list, off_stats, off_bwd, off_bwd_v, total;
@@ -1035,7 +1041,9 @@ bns_status make_nhwc(const bns_shape* sh, const bns_sampling* sp, NhwcProblem& n
     if (np.rows >= 2147483647L) return BNS_ERR_SHAPE;
     const int eb = elem_bytes(pb.dtype);
     np.main = plan_nhwc(pb.C, eb, np.rows, false);
+    np.norm = plan_nhwc(pb.C, eb, np.rows, false, true);
     np.virt = np.main;
+    np.norm_virt = np.norm;
     switch (pb.rule) {
     case BNS_RULE_FULL: np.sampled_rows = np.rows; break;
     case BNS_RULE_BATCH: np.sampled_rows = static_cast<long>(pb.count) * pb.HW; break;
@@ -1043,6 +1051,7 @@ bns_status make_nhwc(const bns_shape* sh, const bns_sampling* sp, NhwcProblem& n
     default:
         np.sampled_rows = static_cast<long>(pb.count) * pb.HW;
         np.virt = plan_nhwc(pb.C, elem_bytes(sp->xv_dtype), np.sampled_rows, false);
+        np.norm_virt = plan_nhwc(pb.C, elem_bytes(sp->xv_dtype), np.sampled_rows, false, true);
         break;
     }
     const int stat_eb = pb.rule == BNS_RULE_VIRTUAL ? elem_bytes(sp->xv_dtype) : eb;
@@ -1143,13 +1152,13 @@ bns_status forward_nhwc_impl(const NhwcProblem& np, const bns_sampling* sp, cons
                           static_cast<float>(1.0 / pb.s), eps, mean, invstd);
     }
     BNS_NHWC_BY_TYPE_V(pb.dtype, pb.C,
-                       (launch_grid(BNS_KERNEL_NORMALIZE, nhwc_normalize_kernel<T, V>, np.main.grid, stream, in<T>(x),
-                                    out<T>(y), gamma, beta, mean, invstd, static_cast<int>(np.rows), np.main.shape)));
+                       (launch_grid(BNS_KERNEL_NORMALIZE, nhwc_normalize_kernel<T, V>, np.norm.grid, stream, in<T>(x),
+                                    out<T>(y), gamma, beta, mean, invstd, static_cast<int>(np.rows), np.norm.shape)));
     if (virt && sp->yv)
         BNS_NHWC_BY_TYPE_V(sp->xv_dtype, pb.C,
-                           (launch_grid(BNS_KERNEL_NORMALIZE, nhwc_normalize_kernel<T, V>, np.virt.grid, stream,
+                           (launch_grid(BNS_KERNEL_NORMALIZE, nhwc_normalize_kernel<T, V>, np.norm_virt.grid, stream,
                                         in<T>(sp->xv), out<T>(sp->yv), gamma, beta, mean, invstd,
-                                        static_cast<int>(np.sampled_rows), np.virt.shape)));
+                                        static_cast<int>(np.sampled_rows), np.norm_virt.shape)));
     return last_error();
 }
 
